@@ -1,0 +1,6 @@
+"""CPU oracle of the selection-resolution path — TEST INFRASTRUCTURE ONLY.
+
+Only `tests/`, the smoke check and the benchmark's CPU-baseline / reference leg may import this
+package.  It shares no code with the CUDA library and never imports it.
+"""
+from .oracle import Oracle, build, STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, FLAG_NO_BYTES, kv_footprint_bytes  # noqa: F401
