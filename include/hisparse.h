@@ -1,0 +1,201 @@
+/*
+ * hisparse.h — C-ABI of the B200-native HiSparse selection-resolution library.
+ *
+ * The library implements one thing: the per-layer selection-resolution hot path of HiSparse, a
+ * hierarchical KV cache for top-k sparse-attention decoding.  For every decode step and layer a
+ * batch of selected logical KV positions per request is resolved against a small fixed-size
+ * per-(request, layer) GPU cache: hits are found, misses evict LRU victims, the missing records
+ * are pulled from pinned host KV history over the host link by the GPU's own threads, and the
+ * table of device slots that a sparse-attention kernel reads is emitted (paper Sec. 3.2-3.5).
+ *
+ * Conventions
+ *   - Every function returns HISPARSE_OK (0) or a negative HISPARSE_E* code; nothing throws.
+ *   - "dev" pointers are device pointers, "host" pointers are host pointers.  `stream` arguments
+ *     are `cudaStream_t` values passed as `void *` (NULL = the legacy default stream).
+ *   - append / resolve / prefetch / gather* only enqueue work; they never synchronise the host
+ *     with the device and keep all step-dependent state (lengths, step counters, miss counts,
+ *     miss plans) in device memory, so a sequence of them can be captured in a CUDA graph and
+ *     replayed.  Create, destroy, status, dump and the probes synchronise.
+ *   - The caller owns the host histories (which must stay pinned, mapped and alive until
+ *     destroy), the selection / slot-table / counter buffers and the streams.  The library owns
+ *     the cache pools and all metadata.
+ *   - One handle is bound to one device and is not thread-safe; use one handle per GPU.
+ */
+#ifndef HISPARSE_H_
+#define HISPARSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hisparse hisparse_t; /* opaque, library-owned */
+
+/* error codes */
+#define HISPARSE_OK 0
+#define HISPARSE_EINVAL (-1)      /* bad argument or geometry (k > B, E % 16, layer out of range ...) */
+#define HISPARSE_ENOTPINNED (-2)  /* a host history is not pinned + device-mapped host memory        */
+#define HISPARSE_ENOMEM (-3)      /* device or host allocation failed                                */
+#define HISPARSE_ECUDA (-4)       /* a CUDA call failed; hisparse_last_cuda_error() has the code      */
+#define HISPARSE_ESTATE (-5)      /* call not valid now (e.g. prefetch of a layer whose anchor has not run) */
+
+/* create flags */
+#define HISPARSE_FLAG_SKIP_IO 1u          /* timing mode of Sec. 4.6's "no-IO oracle": misses are resolved
+                                             in metadata but no record is fetched (cache bytes go stale)   */
+#define HISPARSE_FLAG_DEBUG_VALIDATE 2u   /* after every anchor resolve a checking kernel verifies that the
+                                             page table and the slot array are mutual inverses and that the
+                                             recency order is a permutation; failures set a status bit      */
+#define HISPARSE_FLAG_INLINE_WRITE_THROUGH 4u /* append writes through on the caller's stream instead of
+                                             the library's backup stream                                   */
+
+/* sticky device status bits (hisparse_status) */
+#define HISPARSE_STATUS_OUT_OF_RANGE 1u   /* a selected position was outside [0, len) (and not -1)       */
+#define HISPARSE_STATUS_DUPLICATE 2u      /* a position occurred twice in one row                        */
+#define HISPARSE_STATUS_CAPACITY 4u       /* an append found a request's history full; it was dropped    */
+#define HISPARSE_STATUS_INCONSISTENT 8u   /* DEBUG_VALIDATE found broken metadata                        */
+#define HISPARSE_STATUS_TIMEOUT 16u       /* a bounded device-side wait expired                          */
+
+/* limits */
+#define HISPARSE_MAX_CACHE_SLOTS 16384
+#define HISPARSE_MAX_TOP_K 4096
+
+/*
+ * Geometry of one handle (notation of the paper's Table 2: N_batch, N_l, B, k, W_KV * s).
+ * A "record" is the unit the selector picks: a token's KV (DSA), a block (NSA) or a page (Quest).
+ */
+typedef struct {
+  int32_t num_requests;      /* N: concurrent decode requests, fixed for the handle's life            */
+  int32_t num_layers;        /* L: sparse-attention layers                                            */
+  int32_t layers_per_group;  /* 1: every layer selects for itself.  g > 1: layers [a, a+g) share the
+                                selection of their anchor layer a = multiple of g (Sec. 3.5); L % g == 0 */
+  int32_t cache_slots;       /* B: LRU-managed slots per (request, layer); one more slot per (request,
+                                layer) is reserved for the newest record (Sec. 3.3 step 4)              */
+  int32_t top_k;             /* k: row length of sel / slot_table; 1 <= k <= B                          */
+  int64_t entry_bytes;       /* E: bytes per record, a positive multiple of 16                         */
+  const int64_t *capacity;   /* host [N]: maximum number of records of each request's history          */
+  const int64_t *init_len;   /* host [N]: records already present in the history, <= capacity          */
+  void *const *host_history; /* host [N]: base of each request's history, pinned and device-mapped host
+                                memory (cudaHostAlloc / cudaHostRegister with the Mapped flag), 16-byte
+                                aligned, laid out [L][capacity[r]][E]                                   */
+  int32_t device;            /* CUDA device ordinal                                                    */
+  uint32_t flags;            /* HISPARSE_FLAG_*                                                         */
+  int32_t ctas_per_request;  /* thread blocks (one cluster) that share one request's fetch work;
+                                0 = choose from N and the SM count; otherwise 1, 2, 4 or 8             */
+} hisparse_config_t;
+
+/* Sec. 3.3 step (2) "Admission": reserve the per-layer caches and metadata of N requests.  All
+ * caches start cold.  Validates the geometry (EINVAL) and that every history is pinned and mapped
+ * (ENOTPINNED).  Synchronises. */
+int hisparse_create(const hisparse_config_t *cfg, hisparse_t **out);
+
+/* Releases everything the library owns after waiting for its outstanding work.  Synchronises. */
+int hisparse_destroy(hisparse_t *h);
+
+/* Sec. 3.3 step (4) "Write-through of generated KV": every request appends one record per layer.
+ * new_kv_dev is device memory [N][L][E]; request r's records land at position len[r], which then
+ * grows by one.  The records are placed in the reserved slot of each (request, layer) cache, so
+ * the newest position is always resident, and written through to the host history on the
+ * library's backup stream (on `stream` itself with INLINE_WRITE_THROUGH), ordered by events so
+ * that the host copy is complete before any later fetch can reference it.  new_kv_dev may be
+ * reused as soon as work enqueued on `stream` after this call runs.  A request whose history is
+ * full sets STATUS_CAPACITY and keeps its length. */
+int hisparse_append(hisparse_t *h, const void *new_kv_dev, void *stream);
+
+/* Sec. 3.3 step (3) / Sec. 3.4 (the fused Resolve kernel): resolve `layer` for all N requests in
+ * ONE kernel launch, one thread-block cluster per request.
+ *   sel_dev        int32 [N][k]  selected positions of each request, any order; -1 = padding
+ *   slot_table_dev int32 [N][k]  out: for each selection the index of its record in
+ *                                hisparse_layer_pool(layer), i.e. r*(B+1) + slot with slot in [0, B]
+ *                                (slot B = the reserved newest-record slot); -1 for padding and for
+ *                                out-of-range positions
+ *   hits_dev, misses_dev int32 [N]  out: selections found resident / fetched; hits + misses = number
+ *                                of distinct valid selections of the row
+ * Semantics (deterministic): selections already resident are hits, keep their slot and are stamped
+ * first (recency stamp 2t+1, t = number of resolves of this (request, group) so far); the misses
+ * then take the slots that were not hit, in ascending (stamp, slot) order, the i-th miss of the row
+ * taking the i-th such slot, and are stamped 2t; their records are copied from the host history
+ * into those slots before the kernel ends.  The anchor layer also records its miss plan.
+ * For a shared layer (layer % layers_per_group != 0) sel_dev is ignored: the call waits for that
+ * layer's prefetch (or, if hisparse_prefetch was not called for it since the anchor's resolve,
+ * replays the anchor's plan on `stream`), then emits the anchor's table and counts (Sec. 3.5).
+ * Every layer of a group must be resolved once per step, anchor first.
+ * A position outside [0, len) sets STATUS_OUT_OF_RANGE and yields -1; a position repeated in a row
+ * sets STATUS_DUPLICATE, takes the slot of its first occurrence and is counted once. */
+int hisparse_resolve(hisparse_t *h, int layer, const int32_t *sel_dev, int32_t *slot_table_dev,
+                     int32_t *hits_dev, int32_t *misses_dev, void *stream);
+
+/* Sec. 3.5 "Exact prefetch with shared selections": replay the miss plan recorded by `layer`'s
+ * anchor into `layer`'s cache with a copy-only kernel on side_stream (no probing, no LRU update),
+ * ordered after the anchor's resolve by an event.  `layer` must be a shared layer whose anchor has
+ * been resolved in this step (ESTATE otherwise).  The later hisparse_resolve(layer) waits for it. */
+int hisparse_prefetch(hisparse_t *h, int layer, void *side_stream);
+
+/* Makes `stream` wait for everything the library has in flight on its own backup stream and on
+ * side streams given to hisparse_prefetch.  Needed before ending a stream capture that contains an
+ * append, and before the host reads the histories.  The resolve of the last layer joins the
+ * write-through by itself. */
+int hisparse_join(hisparse_t *h, void *stream);
+
+/* Device base of one layer's cache pool: N*(B+1) records of E bytes (what the attention kernel
+ * gathers from with the slot table).  Valid until destroy. */
+const void *hisparse_layer_pool(const hisparse_t *h, int layer);
+
+/* Stand-in for the sparse-attention consumer (Sec. 3.4 Phase 5: "the downstream gather can read
+ * the selected records directly from the GPU cache"): copies the record of every table entry into
+ * out_dev, uint8 [N][k][E]; entries with table value -1 are zero-filled. */
+int hisparse_gather(hisparse_t *h, int layer, const int32_t *slot_table_dev, void *out_dev, void *stream);
+
+/* Exactness check of Sec. 3.1 ("HiSparse may change where entries reside, not the selected
+ * positions or the outputs"): for every valid selection compares the E bytes its table entry
+ * addresses with the host history's record at that position and adds the number of differing
+ * selections to *mismatches_dev (int32, not cleared).  Joins the write-through first. */
+int hisparse_gather_check(hisparse_t *h, int layer, const int32_t *sel_dev, const int32_t *slot_table_dev,
+                          int32_t *mismatches_dev, void *stream);
+
+/* Sticky status bits accumulated by the device code (HISPARSE_STATUS_*).  Synchronises the device. */
+int hisparse_status(hisparse_t *h, uint32_t *bits);
+int hisparse_clear_status(hisparse_t *h);
+
+/* Copies one (request, layer)'s metadata to host buffers; any pointer may be NULL.  slot_pos [B]
+ * (position held by each slot, -1 = empty), last_use [B] (recency stamps), lru_order [B] (slots from
+ * least to most recent), pos2slot [capacity[req]] (page table, -1 = host-only).  Synchronises. */
+int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, uint32_t *last_use,
+                        int32_t *lru_order, int32_t *pos2slot, int64_t *len, int64_t *newest,
+                        uint32_t *resolves);
+
+/* Miss plan recorded by the last resolve of `layer`'s anchor for request req: plan_pos / plan_slot
+ * are host int32 [k]; *n receives the number of entries.  Synchronises. */
+int hisparse_dump_plan(hisparse_t *h, int req, int layer, int32_t *plan_pos, int32_t *plan_slot, int32_t *n);
+
+/* Device bytes a handle of this geometry allocates: the KV term N*L*(B+1)*E (Sec. 3.1 "Bounded
+ * device footprint", plus the reserved slot) in *kv_bytes and the metadata in *meta_bytes. */
+int hisparse_device_bytes(const hisparse_config_t *cfg, size_t *kv_bytes, size_t *meta_bytes);
+
+/* Launch geometry chosen at create: thread blocks per request and threads per block. */
+int hisparse_launch_geometry(const hisparse_t *h, int32_t *ctas_per_request, int32_t *threads, int32_t *smem_bytes);
+
+/* Pinned + device-mapped host memory for histories (cudaHostAlloc, portable | mapped). */
+int hisparse_host_alloc(size_t bytes, void **out);
+int hisparse_host_free(void *p);
+
+/* Host-link peak: best-of-`reps` bulk cudaMemcpyAsync of `bytes` from pinned host memory to the
+ * device, timed with CUDA events; *gb_per_s = bytes / best time.  Allocates and frees its own
+ * buffers.  Synchronises. */
+int hisparse_host_link_probe(int device, size_t bytes, int reps, double *gb_per_s);
+
+/* Ceiling for thread-issued scattered reads over the host link: a copy-only kernel (no metadata)
+ * fetches `num_records` records of entry_bytes each from pseudo-random record slots of the pinned
+ * buffer host_buf (host_bytes long) into device memory; best-of-`reps` CUDA-event time is returned
+ * as *gb_per_s.  Allocates and frees its own device buffers.  Synchronises. */
+int hisparse_scatter_read_probe(int device, const void *host_buf, size_t host_bytes, int64_t entry_bytes,
+                                int32_t num_records, int32_t num_ctas, int reps, double *gb_per_s);
+
+const char *hisparse_strerror(int code);
+int hisparse_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HISPARSE_H_ */

@@ -1,0 +1,1116 @@
+// HiSparse selection resolution for B200 (sm_100a): kernels and the C-ABI declared in hisparse.h.
+//
+// Data layout in HBM (N requests, L layers in G = L / layers_per_group groups, B slots, k selections,
+// E bytes per record):
+//   pool      uint8  [L][N][B+1][E]   cache pools; slot B of each (r, l) is the reserved newest-record slot
+//   slot_pos  int32  [N][G][B]        position held by each slot, -1 = empty
+//   last_use  uint32 [N][G][B]        recency stamps: 2t+1 hit at resolve t, 2t fetched at resolve t, 0 unused
+//   order     uint16 [N][G][B]        slots from least to most recent; always equal to sorting the slots by
+//                                     (last_use, slot).  Kept so that victim choice is a prefix scan, not a sort
+//   pos2slot  int32  ragged [N][G][capacity[r]]  the page table (Sec. 3.2), -1 = host-only
+//   plan_*    int32  [N][G][k]        miss plan of the last anchor resolve (Sec. 3.5)
+// All step-dependent scalars (resolve counters, number of appends, plan sizes) live in device memory so
+// that every launch is replayable from a CUDA graph.
+//
+// The Resolve kernel (Sec. 3.4, Phases 1-5) runs one thread-block cluster per request.  The cluster's first
+// block does the metadata: it hashes the selected positions into shared memory, probes the position of every
+// slot against that table (coalesced scan of slot_pos), compacts the misses in selection order with
+// ballot/prefix sums, walks the recency order once to split the non-hit slots into the first m (victims) and the
+// rest, and rewrites the order as (untouched ++ victims by slot ++ hits by slot).  After a cluster barrier all
+// blocks of the cluster stream the missing records from pinned host memory into their slots with 16-byte
+// non-coherent loads (Phase 4), so the fetch parallelism does not depend on the number of requests.
+#include "hisparse.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+#define HS_CUDA(call)                                   \
+  do {                                                  \
+    cudaError_t e_ = (call);                            \
+    if (e_ != cudaSuccess) {                            \
+      g_last_cuda_error = (int)e_;                      \
+      return e_ == cudaErrorMemoryAllocation ? HISPARSE_ENOMEM : HISPARSE_ECUDA; \
+    }                                                   \
+  } while (0)
+
+constexpr int kThreads = 1024;       // threads per block of the resolve / replay kernels
+constexpr int kFetchUnroll = 4;      // 16-byte host loads in flight per thread
+constexpr int32_t kMiss = -2;        // s_out marker: valid selection, not (yet) found resident
+constexpr int32_t kDupBase = -3;     // s_out marker: duplicate of row entry -(v + 3)
+
+// Everything a kernel needs, passed by value.
+struct DevState {
+  int N, L, lpg, G, B, k, H, W, hshift;
+  int64_t E;
+  int64_t layer_pool_bytes;
+  uint32_t upe;  // 16-byte units per record
+  uint32_t flags;
+  uint8_t *pool;
+  int32_t *slot_pos;
+  uint32_t *last_use;
+  uint16_t *order;
+  int32_t *pos2slot;
+  const int64_t *cap, *init_len, *p2s_off;
+  uint8_t *const *host;
+  uint32_t *t;
+  int32_t *plan_pos, *plan_slot, *plan_n;
+  int32_t *anchor_out, *anchor_hits, *anchor_misses;
+  int32_t *n_appends;
+  uint32_t *ticket;
+  uint32_t *status;
+};
+
+// ------------------------------------------------------------------------------------------ device helpers
+
+__device__ __forceinline__ uint4 ld_host16(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Multiplicative hash of a position into a table of H = 2^(32 - shift) entries.
+__device__ __forceinline__ uint32_t hash_pos(int32_t p, int shift) {
+  return ((uint32_t)p * 0x9E3779B1u) >> shift;
+}
+
+// Block-wide exclusive prefix count of one flag per thread.  s_warp: 32 ints of scratch.
+__device__ __forceinline__ int block_flag_scan(bool flag, int *s_warp, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const unsigned b = __ballot_sync(0xffffffffu, flag);
+  const int within = __popc(b & ((1u << lane) - 1u));
+  if (lane == 0) s_warp[warp] = __popc(b);
+  __syncthreads();
+  const int v = lane < nw ? s_warp[lane] : 0;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  const int warp_excl = __shfl_sync(0xffffffffu, incl - v, warp);
+  total = __shfl_sync(0xffffffffu, incl, 31);
+  __syncthreads();
+  return warp_excl + within;
+}
+
+__device__ __forceinline__ void history_state(const DevState &d, int r, int64_t &len, int64_t &newest) {
+  const int64_t na = *(volatile int32_t *)d.n_appends;
+  const int64_t il = d.init_len[r], cap = d.cap[r];
+  len = il + na < cap ? il + na : cap;
+  newest = (na > 0 && il + na <= cap) ? il + na - 1 : -1;
+}
+
+// Phase 4 (Sec. 3.4): copy m records host -> cache for request r of `layer`.  The plan (position, slot) is read
+// from shared memory.  The work is flattened into 16-byte units so that consecutive threads read consecutive
+// host addresses across record boundaries; `part` of `nparts` blocks share it.
+__device__ __forceinline__ void fetch_records(const DevState &d, int r, int layer, int m, const int32_t *s_pos,
+                                              const int32_t *s_slot, int part, int nparts) {
+  const uint32_t upe = d.upe;
+  const uint8_t *hbase = d.host[r] + (int64_t)layer * d.cap[r] * d.E;
+  uint8_t *pbase = d.pool + (int64_t)layer * d.layer_pool_bytes + (int64_t)r * (d.B + 1) * d.E;
+  const uint64_t total = (uint64_t)m * upe;
+  const uint64_t stride = (uint64_t)nparts * blockDim.x;
+  for (uint64_t base = (uint64_t)part * blockDim.x + threadIdx.x; base < total; base += stride * kFetchUnroll) {
+    uint4 v[kFetchUnroll];
+    uint8_t *dst[kFetchUnroll];
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i) {
+      const uint64_t u = base + (uint64_t)i * stride;
+      dst[i] = nullptr;
+      if (u < total) {
+        const uint32_t rec = (uint32_t)(u / upe);
+        const uint32_t off = (uint32_t)(u - (uint64_t)rec * upe);
+        v[i] = ld_host16(hbase + ((int64_t)s_pos[rec] * upe + off) * 16);
+        dst[i] = pbase + ((int64_t)s_slot[rec] * upe + off) * 16;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i)
+      if (dst[i]) *reinterpret_cast<uint4 *>(dst[i]) = v[i];
+  }
+}
+
+// ------------------------------------------------------------------------------------------ Resolve (Sec. 3.4)
+
+__global__ void __launch_bounds__(kThreads, 1)
+resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ sel, int32_t *__restrict__ table,
+               int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out, const int S) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ int s_warp[32];
+  __shared__ int s_misc[4];  // [0] any duplicate  [1] valid distinct selections
+  const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  const int r = blockIdx.x / S, part = blockIdx.x - r * S;
+  const int g = layer / d.lpg;
+  const int k = d.k, B = d.B, H = d.H, W = d.W;
+  const int64_t rg = (int64_t)r * d.G + g;
+
+  int32_t *s_sel = reinterpret_cast<int32_t *>(smem_raw);
+  int32_t *s_out = s_sel + k;
+  int32_t *s_plan_pos = s_out + k;   // first the row indices of the misses, then their positions
+  int32_t *s_plan_slot = s_plan_pos + k;  // victims, in order
+  uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_plan_slot + k);
+  uint32_t *s_hitbits = s_tab + H;
+  uint32_t *s_vicbits = s_hitbits + W;
+  int32_t *s_hitpre = reinterpret_cast<int32_t *>(s_vicbits + W);
+  int32_t *s_vicpre = s_hitpre + W;
+  uint16_t *s_order = reinterpret_cast<uint16_t *>(s_vicpre + W);
+
+  int m = 0;
+  if (part == 0) {
+    int64_t len, newest;
+    history_state(d, r, len, newest);
+    const uint32_t t = d.t[rg] + 1u;
+    const uint32_t hit_stamp = 2u * t + 1u, miss_stamp = 2u * t;
+    int32_t *slot_pos = d.slot_pos + rg * B;
+    uint32_t *last_use = d.last_use + rg * B;
+    uint16_t *order = d.order + rg * B;
+    int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
+    const int32_t *row = sel + (int64_t)r * k;
+
+    // Phase 1: stage the selected positions and hash them (value = row index + 1, 0 = empty).
+    for (int i = tid; i < H; i += T) s_tab[i] = 0u;
+    for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
+    if (tid < 4) s_misc[tid] = 0;
+    for (int j = tid; j < k; j += T) s_sel[j] = row[j];
+    __syncthreads();
+
+    uint32_t my_status = 0;
+    int my_valid = 0;
+    for (int j = tid; j < k; j += T) {
+      const int32_t p = s_sel[j];
+      int32_t o = -1;
+      if (p == -1) {
+      } else if (p < 0 || (int64_t)p >= len) {
+        my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
+      } else {
+        o = (int64_t)p == newest ? B : kMiss;
+        ++my_valid;
+        uint32_t hsh = hash_pos(p, d.hshift);
+        for (int it = 0; it < H; ++it) {
+          uint32_t cur = *(volatile uint32_t *)&s_tab[hsh];
+          if (cur == 0u) {
+            cur = atomicCAS(&s_tab[hsh], 0u, (uint32_t)j + 1u);
+            if (cur == 0u) break;
+          }
+          if (s_sel[cur - 1u] == p) {  // the same position again: the lowest row index owns the entry
+            atomicMin(&s_tab[hsh], (uint32_t)j + 1u);
+            s_misc[0] = 1;
+            break;
+          }
+          hsh = (hsh + 1u) & (uint32_t)(H - 1);
+        }
+      }
+      s_out[j] = o;
+    }
+    __syncthreads();
+    if (s_misc[0]) {  // rare: mark every later occurrence of a repeated position
+      for (int j = tid; j < k; j += T) {
+        if (s_out[j] == kMiss || s_out[j] == B) {
+          const int32_t p = s_sel[j];
+          uint32_t hsh = hash_pos(p, d.hshift);
+          for (int it = 0; it < H; ++it) {
+            const uint32_t cur = s_tab[hsh];
+            if (cur == 0u) break;
+            if (s_sel[cur - 1u] == p) {
+              if ((int)cur - 1 != j) {
+                s_out[j] = kDupBase - ((int)cur - 1);
+                --my_valid;
+                my_status |= HISPARSE_STATUS_DUPLICATE;
+              }
+              break;
+            }
+            hsh = (hsh + 1u) & (uint32_t)(H - 1);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) my_valid += __shfl_xor_sync(0xffffffffu, my_valid, o);
+    if (lane == 0 && my_valid) atomicAdd(&s_misc[1], my_valid);
+    __syncthreads();
+
+    // Phase 2: probe the position held by every slot; hits keep their slot and are stamped first.
+    for (int base = 0; base < B; base += T) {
+      const int s = base + tid;
+      bool hit = false;
+      if (s < B) {
+        const int32_t p = slot_pos[s];
+        if (p >= 0) {
+          uint32_t hsh = hash_pos(p, d.hshift);
+          for (int it = 0; it < H; ++it) {
+            const uint32_t cur = s_tab[hsh];
+            if (cur == 0u) break;
+            if (s_sel[cur - 1u] == p) {
+              if (s_out[cur - 1u] == kMiss) {
+                s_out[cur - 1u] = s;
+                hit = true;
+                last_use[s] = hit_stamp;
+              }
+              break;
+            }
+            hsh = (hsh + 1u) & (uint32_t)(H - 1);
+          }
+        }
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, hit);
+      if (lane == 0 && base + warp * 32 < B) s_hitbits[(base >> 5) + warp] = bal;
+    }
+    __syncthreads();
+
+    // Phase 3a: compact the misses in selection order.
+    for (int base = 0; base < k; base += T) {
+      const int j = base + tid;
+      const bool flag = j < k && s_out[j] == kMiss;
+      int total;
+      const int rank = block_flag_scan(flag, s_warp, total);
+      if (flag) s_plan_pos[m + rank] = j;
+      m += total;
+    }
+    // Phase 3b: walk the recency order; the first m slots that were not hit are the victims, in order;
+    // the other non-hit slots keep their relative order at the front of the new order.
+    int n_nonhit = 0;
+    for (int base = 0; base < B; base += T) {
+      const int q = base + tid;
+      int s = 0;
+      bool flag = false;
+      if (q < B) {
+        s = order[q];
+        flag = !((s_hitbits[s >> 5] >> (s & 31)) & 1u);
+      }
+      int total;
+      const int rank = n_nonhit + block_flag_scan(flag, s_warp, total);
+      if (flag) {
+        if (rank < m) {
+          s_plan_slot[rank] = s;
+          atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
+        } else {
+          s_order[rank - m] = (uint16_t)s;
+        }
+      }
+      n_nonhit += total;
+    }
+    __syncthreads();
+    // new order = untouched ++ victims by slot ++ hits by slot: word-level prefix counts, then one pass.
+    if (warp == 0) {
+      int run_h = 0, run_v = 0;
+      for (int wb = 0; wb < W; wb += 32) {
+        const int w = wb + lane;
+        const int ch = w < W ? __popc(s_hitbits[w]) : 0, cv = w < W ? __popc(s_vicbits[w]) : 0;
+        int ih = ch, iv = cv;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int nh = __shfl_up_sync(0xffffffffu, ih, o), nv = __shfl_up_sync(0xffffffffu, iv, o);
+          if (lane >= o) { ih += nh; iv += nv; }
+        }
+        if (w < W) { s_hitpre[w] = run_h + ih - ch; s_vicpre[w] = run_v + iv - cv; }
+        run_h += __shfl_sync(0xffffffffu, ih, 31);
+        run_v += __shfl_sync(0xffffffffu, iv, 31);
+      }
+    }
+    __syncthreads();
+    const int n_surv = n_nonhit - m;
+    for (int s = tid; s < B; s += T) {
+      const int w = s >> 5;
+      const uint32_t bit = 1u << (s & 31), lt = bit - 1u;
+      const uint32_t vw = s_vicbits[w], hw = s_hitbits[w];
+      if (vw & bit) s_order[n_surv + s_vicpre[w] + __popc(vw & lt)] = (uint16_t)s;
+      else if (hw & bit) s_order[n_nonhit + s_hitpre[w] + __popc(hw & lt)] = (uint16_t)s;
+    }
+    // Phase 3c / 5: the i-th miss takes the i-th victim; page table, slot array, stamps, plan.
+    int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
+    for (int i = tid; i < m; i += T) {
+      const int j = s_plan_pos[i];
+      const int v = s_plan_slot[i];
+      const int32_t p = s_sel[j];
+      const int32_t old = slot_pos[v];
+      if (old >= 0) p2s[old] = -1;
+      slot_pos[v] = p;
+      p2s[p] = v;
+      last_use[v] = miss_stamp;
+      s_out[j] = v;
+      plan_pos_g[i] = p;
+      plan_slot_g[i] = v;
+      s_plan_pos[i] = p;
+    }
+    __syncthreads();
+    // Phase 5: publish the slot table in selection order, the new recency order and the counters.
+    int32_t *trow = table + (int64_t)r * k;
+    int32_t *arow = d.anchor_out + rg * k;
+    for (int j = tid; j < k; j += T) {
+      int32_t o = s_out[j];
+      if (o <= kDupBase) o = s_out[kDupBase - o];
+      trow[j] = o < 0 ? -1 : r * (B + 1) + o;
+      if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
+    }
+    for (int q = tid; q < B; q += T) order[q] = s_order[q];
+    if (tid == 0) {
+      const int nvalid = s_misc[1];
+      hits_out[r] = nvalid - m;
+      misses_out[r] = m;
+      d.plan_n[rg] = m;
+      d.anchor_hits[rg] = nvalid - m;
+      d.anchor_misses[rg] = m;
+      d.t[rg] = t;
+    }
+    if (my_status) atomicOr(d.status, my_status);
+  }
+
+  if (S > 1) {
+    __threadfence();
+    cluster_barrier();
+    if (part != 0) {
+      m = __ldcg(d.plan_n + rg);
+      const int32_t *pp = d.plan_pos + rg * k, *ps = d.plan_slot + rg * k;
+      for (int i = tid; i < m; i += T) { s_plan_pos[i] = __ldcg(pp + i); s_plan_slot[i] = __ldcg(ps + i); }
+      __syncthreads();
+    }
+  }
+  // Phase 4: fetch the missing records.
+  if (!(d.flags & HISPARSE_FLAG_SKIP_IO)) fetch_records(d, r, layer, m, s_plan_pos, s_plan_slot, part, S);
+}
+
+// ------------------------------------------------------------------------------------------ plan replay (Sec. 3.5)
+
+// Copy-only kernel: replays the anchor's miss plan into a shared layer's cache.  grid = N * S blocks.
+__global__ void __launch_bounds__(kThreads, 1) replay_kernel(const DevState d, const int layer, const int S) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  int32_t *s_plan_pos = reinterpret_cast<int32_t *>(smem_raw);
+  int32_t *s_plan_slot = s_plan_pos + d.k;
+  const int r = blockIdx.x / S, part = blockIdx.x - r * S;
+  const int64_t rg = (int64_t)r * d.G + layer / d.lpg;
+  const int m = d.plan_n[rg];
+  const int32_t *pp = d.plan_pos + rg * d.k, *ps = d.plan_slot + rg * d.k;
+  for (int i = threadIdx.x; i < m; i += blockDim.x) { s_plan_pos[i] = pp[i]; s_plan_slot[i] = ps[i]; }
+  __syncthreads();
+  if (!(d.flags & HISPARSE_FLAG_SKIP_IO)) fetch_records(d, r, layer, m, s_plan_pos, s_plan_slot, part, S);
+}
+
+// A shared layer reuses its anchor's slot table (same local slots, same request offsets) and counts.
+__global__ void shared_table_kernel(const DevState d, const int layer, int32_t *__restrict__ table,
+                                    int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out) {
+  const int r = blockIdx.x;
+  const int64_t rg = (int64_t)r * d.G + layer / d.lpg;
+  for (int j = threadIdx.x; j < d.k; j += blockDim.x) {
+    const int32_t o = d.anchor_out[rg * d.k + j];
+    table[(int64_t)r * d.k + j] = o < 0 ? -1 : r * (d.B + 1) + o;
+  }
+  if (threadIdx.x == 0) { hits_out[r] = d.anchor_hits[rg]; misses_out[r] = d.anchor_misses[rg]; }
+}
+
+// ------------------------------------------------------------------------------------------ append (Sec. 3.3 step 4)
+
+__device__ __forceinline__ void copy16(uint8_t *dst, const uint8_t *src, uint32_t units) {
+  for (uint32_t u = threadIdx.x; u < units; u += blockDim.x)
+    reinterpret_cast<uint4 *>(dst)[u] = reinterpret_cast<const uint4 *>(src)[u];
+}
+
+// grid = N * L blocks.  Block (r, l) puts request r's new record of layer l into the reserved slot; with
+// write_through != 0 it also stores it into the host history.  The last block to finish bumps the append count.
+__global__ void append_kernel(const DevState d, const uint8_t *__restrict__ new_kv, const int write_through) {
+  const int r = blockIdx.x / d.L, l = blockIdx.x - r * d.L;
+  const int64_t na = *(volatile int32_t *)d.n_appends;
+  const int64_t p = d.init_len[r] + na;
+  if (p < d.cap[r]) {
+    const uint8_t *src = new_kv + ((int64_t)r * d.L + l) * d.E;
+    copy16(d.pool + (int64_t)l * d.layer_pool_bytes + ((int64_t)r * (d.B + 1) + d.B) * d.E, src, d.upe);
+    if (write_through) {
+      copy16(d.host[r] + ((int64_t)l * d.cap[r] + p) * d.E, src, d.upe);
+      __threadfence_system();
+    }
+  } else if (threadIdx.x == 0 && l == 0) {
+    atomicOr(d.status, HISPARSE_STATUS_CAPACITY);
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t prev = atomicAdd(d.ticket, 1u);
+    if (prev == gridDim.x - 1) {
+      *(volatile int32_t *)d.n_appends = (int32_t)na + 1;
+      *(volatile uint32_t *)d.ticket = 0u;
+      __threadfence();
+    }
+  }
+}
+
+// Backup-stream half of the append: reserved slot -> host history at the position just appended.
+__global__ void write_through_kernel(const DevState d) {
+  const int r = blockIdx.x / d.L, l = blockIdx.x - r * d.L;
+  const int64_t na = *(volatile int32_t *)d.n_appends;
+  const int64_t p = d.init_len[r] + na - 1;
+  if (na > 0 && p < d.cap[r]) {
+    copy16(d.host[r] + ((int64_t)l * d.cap[r] + p) * d.E,
+           d.pool + (int64_t)l * d.layer_pool_bytes + ((int64_t)r * (d.B + 1) + d.B) * d.E, d.upe);
+    __threadfence_system();
+  }
+}
+
+// ------------------------------------------------------------------------------------------ consumer stand-ins
+
+// One warp per table entry: out[r][j] = pool[table[r][j]] (zeros for -1).
+__global__ void gather_kernel(const DevState d, const int layer, const int32_t *__restrict__ table,
+                              uint8_t *__restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  const uint8_t *pool = d.pool + (int64_t)layer * d.layer_pool_bytes;
+  for (int64_t e = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); e < (int64_t)d.N * d.k; e += nwarps) {
+    const int32_t s = table[e];
+    uint4 *dst = reinterpret_cast<uint4 *>(out + e * d.E);
+    if (s < 0) {
+      for (uint32_t u = lane; u < d.upe; u += 32) dst[u] = make_uint4(0, 0, 0, 0);
+    } else {
+      const uint4 *src = reinterpret_cast<const uint4 *>(pool + (int64_t)s * d.E);
+      for (uint32_t u = lane; u < d.upe; u += 32) dst[u] = src[u];
+    }
+  }
+}
+
+// One warp per selection: the bytes the table entry addresses must equal the host history's record.
+__global__ void gather_check_kernel(const DevState d, const int layer, const int32_t *__restrict__ sel,
+                                    const int32_t *__restrict__ table, int32_t *mismatches) {
+  const int lane = threadIdx.x & 31;
+  const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  const uint8_t *pool = d.pool + (int64_t)layer * d.layer_pool_bytes;
+  for (int64_t e = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); e < (int64_t)d.N * d.k; e += nwarps) {
+    const int r = (int)(e / d.k);
+    int64_t len, newest;
+    history_state(d, r, len, newest);
+    const int32_t p = sel[e];
+    if (p < 0 || p >= len) continue;
+    const int32_t s = table[e];
+    bool bad = s < r * (d.B + 1) || s > r * (d.B + 1) + d.B;
+    if (!bad) {
+      const uint4 *a = reinterpret_cast<const uint4 *>(pool + (int64_t)s * d.E);
+      const uint8_t *hb = d.host[r] + ((int64_t)layer * d.cap[r] + p) * d.E;
+      for (uint32_t u = lane; u < d.upe; u += 32) {
+        const uint4 x = a[u], y = ld_host16(hb + (int64_t)u * 16);
+        bad |= x.x != y.x || x.y != y.y || x.z != y.z || x.w != y.w;
+      }
+    }
+    bad = __any_sync(0xffffffffu, bad);
+    if (bad && lane == 0) atomicAdd(mismatches, 1);
+  }
+}
+
+// DEBUG_VALIDATE: one block per (request, group).
+__global__ void validate_kernel(const DevState d, const int g) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint32_t *seen = reinterpret_cast<uint32_t *>(smem_raw);
+  const int r = blockIdx.x, B = d.B;
+  const int64_t rg = (int64_t)r * d.G + g;
+  const int32_t *slot_pos = d.slot_pos + rg * B;
+  const uint32_t *last_use = d.last_use + rg * B;
+  const uint16_t *order = d.order + rg * B;
+  const int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
+  for (int i = threadIdx.x; i < d.W; i += blockDim.x) seen[i] = 0u;
+  __syncthreads();
+  bool bad = false;
+  for (int s = threadIdx.x; s < B; s += blockDim.x) {
+    const int32_t p = slot_pos[s];
+    if (p >= 0) bad |= p >= d.cap[r] || p2s[p] != s;
+    else bad |= p != -1;
+  }
+  for (int64_t p = threadIdx.x; p < d.cap[r]; p += blockDim.x) {
+    const int32_t s = p2s[p];
+    if (s >= 0) bad |= s >= B || slot_pos[s] != (int32_t)p;
+    else bad |= s != -1;
+  }
+  for (int q = threadIdx.x; q < B; q += blockDim.x) {
+    const int s = order[q];
+    if (s >= B) { bad = true; continue; }
+    const uint32_t old = atomicOr(&seen[s >> 5], 1u << (s & 31));
+    bad |= (old >> (s & 31)) & 1u;
+    if (q + 1 < B) {
+      const int s2 = order[q + 1];
+      if (s2 < B) {
+        const uint32_t a = last_use[s], b = last_use[s2];
+        bad |= a > b || (a == b && s > s2);
+      }
+    }
+  }
+  if (bad) atomicOr(d.status, HISPARSE_STATUS_INCONSISTENT);
+}
+
+__global__ void init_order_kernel(uint16_t *order, int64_t n, int B) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    order[i] = (uint16_t)(i % B);
+}
+
+// Metadata-free scattered copy used by hisparse_scatter_read_probe.
+__global__ void __launch_bounds__(kThreads, 1)
+scatter_probe_kernel(const uint8_t *__restrict__ host, uint8_t *__restrict__ dst, const int32_t *__restrict__ rec_idx,
+                     int m, uint32_t upe) {
+  const uint64_t total = (uint64_t)m * upe, stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t base = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; base < total; base += stride * kFetchUnroll) {
+    uint4 v[kFetchUnroll];
+    uint8_t *out[kFetchUnroll];
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i) {
+      const uint64_t u = base + (uint64_t)i * stride;
+      out[i] = nullptr;
+      if (u < total) {
+        const uint32_t rec = (uint32_t)(u / upe), off = (uint32_t)(u - (uint64_t)rec * upe);
+        v[i] = ld_host16(host + ((int64_t)rec_idx[rec] * upe + off) * 16);
+        out[i] = dst + u * 16;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kFetchUnroll; ++i)
+      if (out[i]) *reinterpret_cast<uint4 *>(out[i]) = v[i];
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------ host state
+
+struct hisparse {
+  DevState d{};
+  int device = 0;
+  int S = 1, T = kThreads;
+  size_t resolve_smem = 0, replay_smem = 0;
+  std::vector<int64_t> cap, init_len, p2s_off;
+  int64_t p2s_total = 0;
+  // device allocations (owned)
+  std::vector<void *> allocs;
+  int64_t *d_cap = nullptr, *d_init_len = nullptr, *d_p2s_off = nullptr;
+  uint8_t **d_host = nullptr;
+  // streams / events
+  cudaStream_t backup = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_wt = nullptr;
+  bool wt_pending = false;
+  std::vector<cudaEvent_t> ev_plan;   // [G] recorded after each anchor resolve
+  std::vector<cudaEvent_t> ev_pref;   // [L] recorded after each prefetch replay
+  std::vector<uint8_t> anchor_done;   // [G] the anchor has been resolved at least once
+  std::vector<uint8_t> replayed;      // [L] plan replayed (or being replayed) since the anchor's last resolve
+  std::vector<uint8_t> pref_unjoined; // [L] a side-stream replay that no stream has waited for yet
+};
+
+namespace {
+
+template <typename T>
+int dev_alloc(hisparse *h, T **out, size_t count) {
+  void *p = nullptr;
+  HS_CUDA(cudaMalloc(&p, std::max<size_t>(count, 1) * sizeof(T)));
+  h->allocs.push_back(p);
+  *out = static_cast<T *>(p);
+  return HISPARSE_OK;
+}
+
+int validate_config(const hisparse_config_t *c) {
+  if (!c) return HISPARSE_EINVAL;
+  if (c->num_requests < 1 || c->num_layers < 1 || c->layers_per_group < 1) return HISPARSE_EINVAL;
+  if (c->num_layers % c->layers_per_group) return HISPARSE_EINVAL;
+  if (c->top_k < 1 || c->top_k > HISPARSE_MAX_TOP_K) return HISPARSE_EINVAL;
+  if (c->cache_slots < c->top_k || c->cache_slots > HISPARSE_MAX_CACHE_SLOTS) return HISPARSE_EINVAL;
+  if (c->entry_bytes < 16 || c->entry_bytes % 16) return HISPARSE_EINVAL;
+  if (c->entry_bytes / 16 > 0x7fffffff) return HISPARSE_EINVAL;
+  if (!c->capacity || !c->init_len) return HISPARSE_EINVAL;
+  for (int r = 0; r < c->num_requests; ++r) {
+    if (c->capacity[r] < 1 || c->capacity[r] > 0x7fffffffLL) return HISPARSE_EINVAL;
+    if (c->init_len[r] < 0 || c->init_len[r] > c->capacity[r]) return HISPARSE_EINVAL;
+  }
+  const int s = c->ctas_per_request;
+  if (!(s == 0 || s == 1 || s == 2 || s == 4 || s == 8)) return HISPARSE_EINVAL;
+  return HISPARSE_OK;
+}
+
+int hash_size(int k) {
+  int H = 32;
+  while (H < 2 * k) H <<= 1;
+  return H;
+}
+
+size_t resolve_smem_bytes(int B, int k) {
+  const int H = hash_size(k), W = (B + 31) / 32;
+  return (size_t)4 * k * 4 + (size_t)H * 4 + (size_t)4 * W * 4 + (size_t)B * 2;
+}
+
+cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
+
+int launch_resolve(hisparse *h, int layer, const int32_t *sel, int32_t *table, int32_t *hits, int32_t *misses,
+                   cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(h->d.N * h->S));
+  cfg.blockDim = dim3((unsigned)h->T);
+  cfg.dynamicSmemBytes = h->resolve_smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)h->S;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel, h->d, layer, sel, table, hits, misses, h->S));
+  return HISPARSE_OK;
+}
+
+int launch_replay(hisparse *h, int layer, cudaStream_t st) {
+  replay_kernel<<<h->d.N * h->S, h->T, h->replay_smem, st>>>(h->d, layer, h->S);
+  HS_CUDA(cudaGetLastError());
+  return HISPARSE_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------ C-ABI
+
+extern "C" {
+
+const char *hisparse_strerror(int code) {
+  switch (code) {
+    case HISPARSE_OK: return "ok";
+    case HISPARSE_EINVAL: return "invalid argument or geometry";
+    case HISPARSE_ENOTPINNED: return "host history is not pinned, device-mapped host memory";
+    case HISPARSE_ENOMEM: return "out of memory";
+    case HISPARSE_ECUDA: return "CUDA call failed";
+    case HISPARSE_ESTATE: return "call not valid in the current state";
+    default: return "unknown error";
+  }
+}
+
+int hisparse_last_cuda_error(void) { return g_last_cuda_error; }
+
+int hisparse_device_bytes(const hisparse_config_t *c, size_t *kv_bytes, size_t *meta_bytes) {
+  const int rc = validate_config(c);
+  if (rc) return rc;
+  const size_t N = c->num_requests, L = c->num_layers, G = L / c->layers_per_group, B = c->cache_slots, k = c->top_k;
+  if (kv_bytes) *kv_bytes = N * L * (B + 1) * (size_t)c->entry_bytes;
+  if (meta_bytes) {
+    size_t cap_sum = 0;
+    for (size_t r = 0; r < N; ++r) cap_sum += (size_t)c->capacity[r];
+    *meta_bytes = N * G * B * (4 + 4 + 2)          /* slot_pos, last_use, order */
+                  + cap_sum * G * 4                 /* page tables */
+                  + N * G * k * 4 * 3               /* plan_pos, plan_slot, anchor_out */
+                  + N * G * 4 * 4                   /* t, plan_n, anchor hits / misses */
+                  + N * (8 * 3 + 8) + 16;           /* cap, init_len, p2s_off, host pointers, scalars */
+  }
+  return HISPARSE_OK;
+}
+
+int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
+  if (!out) return HISPARSE_EINVAL;
+  *out = nullptr;
+  int rc = validate_config(c);
+  if (rc) return rc;
+  if (!c->host_history) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(c->device));
+  const int N = c->num_requests, L = c->num_layers, G = L / c->layers_per_group, B = c->cache_slots, k = c->top_k;
+
+  std::vector<uint8_t *> host_dev(N);
+  for (int r = 0; r < N; ++r) {
+    if (!c->host_history[r] || ((uintptr_t)c->host_history[r] & 15)) return HISPARSE_EINVAL;
+    cudaPointerAttributes a;
+    cudaError_t e = cudaPointerGetAttributes(&a, c->host_history[r]);
+    if (e != cudaSuccess) { cudaGetLastError(); return HISPARSE_ENOTPINNED; }
+    if (a.type != cudaMemoryTypeHost || !a.devicePointer) return HISPARSE_ENOTPINNED;
+    host_dev[r] = static_cast<uint8_t *>(a.devicePointer);
+  }
+
+  hisparse *h = new (std::nothrow) hisparse();
+  if (!h) return HISPARSE_ENOMEM;
+  auto fail = [&](int code) { hisparse_destroy(h); return code; };
+  h->device = c->device;
+  DevState &d = h->d;
+  d.N = N; d.L = L; d.lpg = c->layers_per_group; d.G = G; d.B = B; d.k = k;
+  d.H = hash_size(k); d.W = (B + 31) / 32;
+  d.hshift = 32;
+  for (int x = d.H; x > 1; x >>= 1) --d.hshift;
+  d.E = c->entry_bytes; d.upe = (uint32_t)(c->entry_bytes / 16); d.flags = c->flags;
+  d.layer_pool_bytes = (int64_t)N * (B + 1) * d.E;
+  h->cap.assign(c->capacity, c->capacity + N);
+  h->init_len.assign(c->init_len, c->init_len + N);
+  h->p2s_off.resize(N);
+  int64_t off = 0;
+  for (int r = 0; r < N; ++r) { h->p2s_off[r] = off; off += h->cap[r] * G; }
+  h->p2s_total = off;
+
+  h->resolve_smem = resolve_smem_bytes(B, k);
+  h->replay_smem = (size_t)2 * k * 4;
+  int max_optin = 0;
+  if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  if (h->resolve_smem + 1024 > (size_t)max_optin) return fail(HISPARSE_EINVAL);
+  if (cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  if (cudaFuncSetAttribute(replay_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
+
+  // Blocks per request: as many as still let all N clusters be resident at once.
+  if (c->ctas_per_request) {
+    h->S = c->ctas_per_request;
+  } else {
+    h->S = 1;
+    for (int s = 8; s > 1; s >>= 1) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(N * s));
+      cfg.blockDim = dim3(kThreads);
+      cfg.dynamicSmemBytes = h->resolve_smem;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = (unsigned)s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      int nclusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&nclusters, resolve_kernel, &cfg) == cudaSuccess && nclusters >= N) { h->S = s; break; }
+      cudaGetLastError();
+    }
+  }
+
+#define HS_TRY(expr) do { int rc_ = (expr); if (rc_) return fail(rc_); } while (0)
+  const size_t NG = (size_t)N * G;
+  HS_TRY(dev_alloc(h, &d.pool, (size_t)L * d.layer_pool_bytes));
+  HS_TRY(dev_alloc(h, &d.slot_pos, NG * B));
+  HS_TRY(dev_alloc(h, &d.last_use, NG * B));
+  HS_TRY(dev_alloc(h, &d.order, NG * B));
+  HS_TRY(dev_alloc(h, &d.pos2slot, (size_t)h->p2s_total));
+  HS_TRY(dev_alloc(h, &h->d_cap, (size_t)N));
+  HS_TRY(dev_alloc(h, &h->d_init_len, (size_t)N));
+  HS_TRY(dev_alloc(h, &h->d_p2s_off, (size_t)N));
+  HS_TRY(dev_alloc(h, &h->d_host, (size_t)N));
+  HS_TRY(dev_alloc(h, &d.t, NG));
+  HS_TRY(dev_alloc(h, &d.plan_pos, NG * k));
+  HS_TRY(dev_alloc(h, &d.plan_slot, NG * k));
+  HS_TRY(dev_alloc(h, &d.plan_n, NG));
+  HS_TRY(dev_alloc(h, &d.anchor_out, NG * k));
+  HS_TRY(dev_alloc(h, &d.anchor_hits, NG));
+  HS_TRY(dev_alloc(h, &d.anchor_misses, NG));
+  HS_TRY(dev_alloc(h, &d.n_appends, 1));
+  HS_TRY(dev_alloc(h, &d.ticket, 1));
+  HS_TRY(dev_alloc(h, &d.status, 1));
+#undef HS_TRY
+  d.cap = h->d_cap; d.init_len = h->d_init_len; d.p2s_off = h->d_p2s_off; d.host = h->d_host;
+
+#define HS_TRYC(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { g_last_cuda_error = (int)e_; return fail(HISPARSE_ECUDA); } } while (0)
+  HS_TRYC(cudaMemcpy(h->d_cap, h->cap.data(), sizeof(int64_t) * N, cudaMemcpyHostToDevice));
+  HS_TRYC(cudaMemcpy(h->d_init_len, h->init_len.data(), sizeof(int64_t) * N, cudaMemcpyHostToDevice));
+  HS_TRYC(cudaMemcpy(h->d_p2s_off, h->p2s_off.data(), sizeof(int64_t) * N, cudaMemcpyHostToDevice));
+  HS_TRYC(cudaMemcpy(h->d_host, host_dev.data(), sizeof(uint8_t *) * N, cudaMemcpyHostToDevice));
+  HS_TRYC(cudaMemset(d.pool, 0, (size_t)L * d.layer_pool_bytes));
+  HS_TRYC(cudaMemset(d.slot_pos, 0xff, NG * B * 4));
+  HS_TRYC(cudaMemset(d.last_use, 0, NG * B * 4));
+  HS_TRYC(cudaMemset(d.pos2slot, 0xff, (size_t)h->p2s_total * 4));
+  HS_TRYC(cudaMemset(d.t, 0, NG * 4));
+  HS_TRYC(cudaMemset(d.plan_n, 0, NG * 4));
+  HS_TRYC(cudaMemset(d.anchor_out, 0xff, NG * k * 4));
+  HS_TRYC(cudaMemset(d.anchor_hits, 0, NG * 4));
+  HS_TRYC(cudaMemset(d.anchor_misses, 0, NG * 4));
+  HS_TRYC(cudaMemset(d.n_appends, 0, 4));
+  HS_TRYC(cudaMemset(d.ticket, 0, 4));
+  HS_TRYC(cudaMemset(d.status, 0, 4));
+  init_order_kernel<<<296, 256>>>(d.order, (int64_t)NG * B, B);
+  HS_TRYC(cudaGetLastError());
+
+  HS_TRYC(cudaStreamCreateWithFlags(&h->backup, cudaStreamNonBlocking));
+  HS_TRYC(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+  HS_TRYC(cudaEventCreateWithFlags(&h->ev_wt, cudaEventDisableTiming));
+  h->ev_plan.assign(G, nullptr);
+  h->ev_pref.assign(L, nullptr);
+  for (int g = 0; g < G; ++g) HS_TRYC(cudaEventCreateWithFlags(&h->ev_plan[g], cudaEventDisableTiming));
+  for (int l = 0; l < L; ++l) HS_TRYC(cudaEventCreateWithFlags(&h->ev_pref[l], cudaEventDisableTiming));
+  h->anchor_done.assign(G, 0);
+  h->replayed.assign(L, 0);
+  h->pref_unjoined.assign(L, 0);
+  HS_TRYC(cudaDeviceSynchronize());
+#undef HS_TRYC
+  *out = h;
+  return HISPARSE_OK;
+}
+
+int hisparse_destroy(hisparse_t *h) {
+  if (!h) return HISPARSE_EINVAL;
+  cudaSetDevice(h->device);
+  cudaDeviceSynchronize();
+  for (cudaEvent_t e : h->ev_plan) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_pref) if (e) cudaEventDestroy(e);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_wt) cudaEventDestroy(h->ev_wt);
+  if (h->backup) cudaStreamDestroy(h->backup);
+  for (void *p : h->allocs) cudaFree(p);
+  delete h;
+  return HISPARSE_OK;
+}
+
+int hisparse_join(hisparse_t *h, void *stream) {
+  if (!h) return HISPARSE_EINVAL;
+  cudaStream_t st = as_stream(stream);
+  if (h->wt_pending) {
+    HS_CUDA(cudaStreamWaitEvent(st, h->ev_wt, 0));
+    h->wt_pending = false;
+  }
+  for (int l = 0; l < h->d.L; ++l)
+    if (h->pref_unjoined[l]) {
+      HS_CUDA(cudaStreamWaitEvent(st, h->ev_pref[l], 0));
+      h->pref_unjoined[l] = 0;
+    }
+  return HISPARSE_OK;
+}
+
+int hisparse_append(hisparse_t *h, const void *new_kv_dev, void *stream) {
+  if (!h || !new_kv_dev) return HISPARSE_EINVAL;
+  cudaStream_t st = as_stream(stream);
+  const bool inline_wt = h->d.flags & HISPARSE_FLAG_INLINE_WRITE_THROUGH;
+  if (h->wt_pending) {  // the previous write-through still reads the reserved slots
+    HS_CUDA(cudaStreamWaitEvent(st, h->ev_wt, 0));
+    h->wt_pending = false;
+  }
+  append_kernel<<<h->d.N * h->d.L, 256, 0, st>>>(h->d, static_cast<const uint8_t *>(new_kv_dev), inline_wt ? 1 : 0);
+  HS_CUDA(cudaGetLastError());
+  if (!inline_wt) {
+    HS_CUDA(cudaEventRecord(h->ev_fork, st));
+    HS_CUDA(cudaStreamWaitEvent(h->backup, h->ev_fork, 0));
+    write_through_kernel<<<h->d.N * h->d.L, 256, 0, h->backup>>>(h->d);
+    HS_CUDA(cudaGetLastError());
+    HS_CUDA(cudaEventRecord(h->ev_wt, h->backup));
+    h->wt_pending = true;
+  }
+  return HISPARSE_OK;
+}
+
+int hisparse_resolve(hisparse_t *h, int layer, const int32_t *sel_dev, int32_t *slot_table_dev, int32_t *hits_dev,
+                     int32_t *misses_dev, void *stream) {
+  if (!h || layer < 0 || layer >= h->d.L || !slot_table_dev || !hits_dev || !misses_dev) return HISPARSE_EINVAL;
+  cudaStream_t st = as_stream(stream);
+  const int lpg = h->d.lpg, g = layer / lpg;
+  int rc = HISPARSE_OK;
+  if (layer % lpg == 0) {
+    if (!sel_dev) return HISPARSE_EINVAL;
+    // replays of the previous plan of this group must be over before the plan is overwritten
+    for (int l = layer + 1; l < layer + lpg; ++l)
+      if (h->pref_unjoined[l]) {
+        HS_CUDA(cudaStreamWaitEvent(st, h->ev_pref[l], 0));
+        h->pref_unjoined[l] = 0;
+      }
+    rc = launch_resolve(h, layer, sel_dev, slot_table_dev, hits_dev, misses_dev, st);
+    if (rc) return rc;
+    if (lpg > 1) {
+      HS_CUDA(cudaEventRecord(h->ev_plan[g], st));
+      for (int l = layer + 1; l < layer + lpg; ++l) h->replayed[l] = 0;
+    }
+    h->anchor_done[g] = 1;
+    if (h->d.flags & HISPARSE_FLAG_DEBUG_VALIDATE) {
+      validate_kernel<<<h->d.N, 256, (size_t)h->d.W * 4, st>>>(h->d, g);
+      HS_CUDA(cudaGetLastError());
+    }
+  } else {
+    if (!h->anchor_done[g]) return HISPARSE_ESTATE;
+    if (h->pref_unjoined[layer]) {
+      HS_CUDA(cudaStreamWaitEvent(st, h->ev_pref[layer], 0));
+      h->pref_unjoined[layer] = 0;
+    } else if (!h->replayed[layer]) {  // no prefetch was issued: synchronous swap-in on the caller's stream
+      rc = launch_replay(h, layer, st);
+      if (rc) return rc;
+      h->replayed[layer] = 1;
+    }
+    shared_table_kernel<<<h->d.N, 256, 0, st>>>(h->d, layer, slot_table_dev, hits_dev, misses_dev);
+    HS_CUDA(cudaGetLastError());
+  }
+  if (layer == h->d.L - 1 && h->wt_pending) {
+    HS_CUDA(cudaStreamWaitEvent(st, h->ev_wt, 0));
+    h->wt_pending = false;
+  }
+  return HISPARSE_OK;
+}
+
+int hisparse_prefetch(hisparse_t *h, int layer, void *side_stream) {
+  if (!h || layer < 0 || layer >= h->d.L || layer % h->d.lpg == 0) return HISPARSE_EINVAL;
+  const int g = layer / h->d.lpg;
+  if (!h->anchor_done[g]) return HISPARSE_ESTATE;
+  if (h->replayed[layer]) return HISPARSE_OK;
+  cudaStream_t st = as_stream(side_stream);
+  HS_CUDA(cudaStreamWaitEvent(st, h->ev_plan[g], 0));
+  const int rc = launch_replay(h, layer, st);
+  if (rc) return rc;
+  HS_CUDA(cudaEventRecord(h->ev_pref[layer], st));
+  h->replayed[layer] = 1;
+  h->pref_unjoined[layer] = 1;
+  return HISPARSE_OK;
+}
+
+const void *hisparse_layer_pool(const hisparse_t *h, int layer) {
+  if (!h || layer < 0 || layer >= h->d.L) return nullptr;
+  return h->d.pool + (int64_t)layer * h->d.layer_pool_bytes;
+}
+
+int hisparse_gather(hisparse_t *h, int layer, const int32_t *slot_table_dev, void *out_dev, void *stream) {
+  if (!h || layer < 0 || layer >= h->d.L || !slot_table_dev || !out_dev) return HISPARSE_EINVAL;
+  gather_kernel<<<592, 256, 0, as_stream(stream)>>>(h->d, layer, slot_table_dev, static_cast<uint8_t *>(out_dev));
+  HS_CUDA(cudaGetLastError());
+  return HISPARSE_OK;
+}
+
+int hisparse_gather_check(hisparse_t *h, int layer, const int32_t *sel_dev, const int32_t *slot_table_dev,
+                          int32_t *mismatches_dev, void *stream) {
+  if (!h || layer < 0 || layer >= h->d.L || !sel_dev || !slot_table_dev || !mismatches_dev) return HISPARSE_EINVAL;
+  const int rc = hisparse_join(h, stream);
+  if (rc) return rc;
+  // a shared layer is compared against its own history; the selections are its anchor's
+  gather_check_kernel<<<592, 256, 0, as_stream(stream)>>>(h->d, layer, sel_dev, slot_table_dev, mismatches_dev);
+  HS_CUDA(cudaGetLastError());
+  return HISPARSE_OK;
+}
+
+int hisparse_status(hisparse_t *h, uint32_t *bits) {
+  if (!h || !bits) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  HS_CUDA(cudaMemcpy(bits, h->d.status, 4, cudaMemcpyDeviceToHost));
+  return HISPARSE_OK;
+}
+
+int hisparse_clear_status(hisparse_t *h) {
+  if (!h) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  HS_CUDA(cudaMemset(h->d.status, 0, 4));
+  return HISPARSE_OK;
+}
+
+int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, uint32_t *last_use, int32_t *lru_order,
+                        int32_t *pos2slot, int64_t *len, int64_t *newest, uint32_t *resolves) {
+  if (!h || req < 0 || req >= h->d.N || layer < 0 || layer >= h->d.L) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  const int B = h->d.B, g = layer / h->d.lpg;
+  const int64_t rg = (int64_t)req * h->d.G + g;
+  if (slot_pos) HS_CUDA(cudaMemcpy(slot_pos, h->d.slot_pos + rg * B, (size_t)B * 4, cudaMemcpyDeviceToHost));
+  if (last_use) HS_CUDA(cudaMemcpy(last_use, h->d.last_use + rg * B, (size_t)B * 4, cudaMemcpyDeviceToHost));
+  if (lru_order) {
+    std::vector<uint16_t> tmp(B);
+    HS_CUDA(cudaMemcpy(tmp.data(), h->d.order + rg * B, (size_t)B * 2, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < B; ++i) lru_order[i] = tmp[i];
+  }
+  if (pos2slot)
+    HS_CUDA(cudaMemcpy(pos2slot, h->d.pos2slot + h->p2s_off[req] + (int64_t)g * h->cap[req], (size_t)h->cap[req] * 4,
+                       cudaMemcpyDeviceToHost));
+  int32_t na = 0;
+  HS_CUDA(cudaMemcpy(&na, h->d.n_appends, 4, cudaMemcpyDeviceToHost));
+  const int64_t il = h->init_len[req], cap = h->cap[req];
+  if (len) *len = std::min(il + na, cap);
+  if (newest) *newest = (na > 0 && il + na <= cap) ? il + na - 1 : -1;
+  if (resolves) HS_CUDA(cudaMemcpy(resolves, h->d.t + rg, 4, cudaMemcpyDeviceToHost));
+  return HISPARSE_OK;
+}
+
+int hisparse_dump_plan(hisparse_t *h, int req, int layer, int32_t *plan_pos, int32_t *plan_slot, int32_t *n) {
+  if (!h || req < 0 || req >= h->d.N || layer < 0 || layer >= h->d.L || !n) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  const int64_t rg = (int64_t)req * h->d.G + layer / h->d.lpg;
+  HS_CUDA(cudaMemcpy(n, h->d.plan_n + rg, 4, cudaMemcpyDeviceToHost));
+  if (plan_pos) HS_CUDA(cudaMemcpy(plan_pos, h->d.plan_pos + rg * h->d.k, (size_t)h->d.k * 4, cudaMemcpyDeviceToHost));
+  if (plan_slot) HS_CUDA(cudaMemcpy(plan_slot, h->d.plan_slot + rg * h->d.k, (size_t)h->d.k * 4, cudaMemcpyDeviceToHost));
+  return HISPARSE_OK;
+}
+
+int hisparse_launch_geometry(const hisparse_t *h, int32_t *ctas_per_request, int32_t *threads, int32_t *smem_bytes) {
+  if (!h) return HISPARSE_EINVAL;
+  if (ctas_per_request) *ctas_per_request = h->S;
+  if (threads) *threads = h->T;
+  if (smem_bytes) *smem_bytes = (int32_t)h->resolve_smem;
+  return HISPARSE_OK;
+}
+
+int hisparse_host_alloc(size_t bytes, void **out) {
+  if (!out || !bytes) return HISPARSE_EINVAL;
+  *out = nullptr;
+  cudaError_t e = cudaHostAlloc(out, bytes, cudaHostAllocPortable | cudaHostAllocMapped);
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; cudaGetLastError(); return HISPARSE_ENOMEM; }
+  return HISPARSE_OK;
+}
+
+int hisparse_host_free(void *p) {
+  if (!p) return HISPARSE_EINVAL;
+  HS_CUDA(cudaFreeHost(p));
+  return HISPARSE_OK;
+}
+
+int hisparse_host_link_probe(int device, size_t bytes, int reps, double *gb_per_s) {
+  if (!gb_per_s || !bytes || reps < 1) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(device));
+  void *hbuf = nullptr, *dbuf = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  int rc = HISPARSE_OK;
+  float best = 0.f;
+  cudaError_t e = cudaHostAlloc(&hbuf, bytes, cudaHostAllocPortable);
+  if (e == cudaSuccess) e = cudaMalloc(&dbuf, bytes);
+  if (e == cudaSuccess) { memset(hbuf, 0x5a, bytes); e = cudaEventCreate(&e0); }
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  for (int i = 0; e == cudaSuccess && i < reps + 1; ++i) {  // the first pass is a warm-up
+    cudaEventRecord(e0, nullptr);
+    e = cudaMemcpyAsync(dbuf, hbuf, bytes, cudaMemcpyHostToDevice, nullptr);
+    cudaEventRecord(e1, nullptr);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (e == cudaSuccess && i > 0 && (best == 0.f || ms < best)) best = ms;
+  }
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; cudaGetLastError(); rc = e == cudaErrorMemoryAllocation ? HISPARSE_ENOMEM : HISPARSE_ECUDA; }
+  else *gb_per_s = (double)bytes / ((double)best * 1e6);
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (dbuf) cudaFree(dbuf);
+  if (hbuf) cudaFreeHost(hbuf);
+  return rc;
+}
+
+int hisparse_scatter_read_probe(int device, const void *host_buf, size_t host_bytes, int64_t entry_bytes,
+                                int32_t num_records, int32_t num_ctas, int reps, double *gb_per_s) {
+  if (!gb_per_s || !host_buf || entry_bytes < 16 || entry_bytes % 16 || num_records < 1 || num_ctas < 1 || reps < 1)
+    return HISPARSE_EINVAL;
+  const size_t slots = host_bytes / (size_t)entry_bytes;
+  if (slots < 1 || slots > 0x7fffffffu) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(device));
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, host_buf) != cudaSuccess || a.type != cudaMemoryTypeHost || !a.devicePointer) {
+    cudaGetLastError();
+    return HISPARSE_ENOTPINNED;
+  }
+  std::vector<int32_t> idx(num_records);
+  uint64_t s = 0x2545F4914F6CDD1Dull;
+  for (int i = 0; i < num_records; ++i) {
+    s ^= s << 13; s ^= s >> 7; s ^= s << 17;
+    idx[i] = (int32_t)(s % slots);
+  }
+  int32_t *d_idx = nullptr;
+  uint8_t *d_dst = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  float best = 0.f;
+  cudaError_t e = cudaMalloc(&d_idx, (size_t)num_records * 4);
+  if (e == cudaSuccess) e = cudaMalloc(&d_dst, (size_t)num_records * entry_bytes);
+  if (e == cudaSuccess) e = cudaMemcpy(d_idx, idx.data(), (size_t)num_records * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  for (int i = 0; e == cudaSuccess && i < reps + 2; ++i) {
+    cudaEventRecord(e0, nullptr);
+    scatter_probe_kernel<<<num_ctas, kThreads>>>(static_cast<const uint8_t *>(a.devicePointer), d_dst, d_idx, num_records,
+                                                 (uint32_t)(entry_bytes / 16));
+    cudaEventRecord(e1, nullptr);
+    e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (e == cudaSuccess && i >= 2 && (best == 0.f || ms < best)) best = ms;
+  }
+  int rc = HISPARSE_OK;
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; cudaGetLastError(); rc = e == cudaErrorMemoryAllocation ? HISPARSE_ENOMEM : HISPARSE_ECUDA; }
+  else *gb_per_s = (double)num_records * (double)entry_bytes / ((double)best * 1e6);
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (d_dst) cudaFree(d_dst);
+  if (d_idx) cudaFree(d_idx);
+  return rc;
+}
+
+}  // extern "C"

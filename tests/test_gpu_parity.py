@@ -1,0 +1,281 @@
+"""Parity of the CUDA path (called through the C-ABI binding) with the CPU oracle: bit-exact slot
+tables, hit/miss counts, LRU state after every step, miss plans and cache bytes."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_07009_b200 import inputs, hisparse as hs
+from paper_2608_07009_b200 import HiSparse, HostHistory, HiSparseError
+from gpu_harness import Pair, run_trace
+
+pytestmark = pytest.mark.gpu
+
+
+def tiny_workload(N, L, lpg, k, B, E, lens, steps=40):
+    return inputs.Workload("tiny", inputs.KIND_DSA_MIX, N, L, lpg, k, B, E, list(lens), steps)
+
+
+# ------------------------------------------------------------------ tiny-case matrix
+
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 7, 8, 12])
+def test_tiny_matrix(B):
+    rng = np.random.default_rng(100 + B)
+    ks = sorted({1, max(1, B // 2), B})
+    for k in ks:
+        for universe, pad, with_append, E in ((k, 0.0, False, 16), (B + 1, 0.25, True, 48),
+                                              (3 * B, 0.0, True, 1152), (2 * B, 0.2, False, 16)):
+            N = 3
+            lens = [universe, universe + 1, universe + 5]
+            w = tiny_workload(N, 1, 1, k, B, E, lens)
+            pair = Pair(w)
+            prev_newest = [-1] * N
+            try:
+                for step in range(40):
+                    if with_append and step % 2 == 1:
+                        pair.append()
+                    rows = []
+                    for r in range(N):
+                        cur = pair.oracle.length(r)
+                        row = inputs.random_rows(rng, 1, k, cur, pad)[0]
+                        newest = pair.oracle.newest(r)
+                        if with_append and newest >= 0 and step % 3 == 0:
+                            forced = [p for p in dict.fromkeys((newest, prev_newest[r])) if p >= 0][:k]
+                            keep = [p for p in row.tolist() if p not in forced][: k - len(forced)]
+                            row = np.array(forced + keep + [-1] * (k - len(forced) - len(keep)), dtype=np.int32)
+                        prev_newest[r] = newest
+                        rows.append(row)
+                    pair.resolve_and_compare(0, np.stack(rows))
+                    pair.compare_state(0)
+                    if step % 8 == 0:
+                        pair.compare_whole_pool(0)
+                pair.finish()
+            finally:
+                pair.close()
+
+
+@pytest.mark.parametrize("lpg,use_prefetch", [(2, True), (2, False), (4, True), (4, False)])
+def test_shared_groups_tiny(lpg, use_prefetch):
+    rng = np.random.default_rng(lpg)
+    L = 2 * lpg
+    w = tiny_workload(3, L, lpg, 6, 10, 48, [40, 50, 60], steps=16)
+    pair = Pair(w)
+    side = torch.cuda.Stream() if use_prefetch else None
+    try:
+        for step in range(16):
+            pair.append()
+            for a in range(0, L, lpg):
+                sel = np.stack([inputs.random_rows(rng, 1, 6, pair.oracle.length(r))[0] for r in range(3)])
+                for l in range(a, a + lpg):
+                    pair.resolve_and_compare(l, sel, side_stream=side)
+                    pair.compare_state(l)
+                    pair.compare_whole_pool(l)
+        pair.finish()
+    finally:
+        pair.close()
+
+
+# ------------------------------------------------------------------ degenerate rows
+
+def test_all_padding_out_of_range_and_duplicates():
+    w = tiny_workload(2, 1, 1, 4, 6, 32, [20, 30])
+    pair = Pair(w)
+    try:
+        pair.resolve_and_compare(0, np.array([[1, 2, 3, 4], [5, 6, 7, 8]]))
+        pair.resolve_and_compare(0, np.full((2, 4), -1))
+        pair.compare_state(0)
+        pair.finish(0)
+        pair.resolve_and_compare(0, np.array([[1, 20, -9, 2], [29, 30, 5, 1000000]]))
+        pair.compare_state(0)
+        pair.finish(hs.STATUS_OUT_OF_RANGE)
+        pair.gpu.clear_status()
+        pair.oracle.clear_status()
+        pair.resolve_and_compare(0, np.array([[9, 4, 9, 4], [7, 7, 7, 7]]))
+        pair.resolve_and_compare(0, np.array([[4, 4, 9, 10], [-1, 7, 11, 7]]))
+        pair.compare_state(0)
+        pair.finish(hs.STATUS_DUPLICATE)
+    finally:
+        pair.close()
+
+
+def test_k_equals_b_all_miss_every_step():
+    k = B = 64
+    w = tiny_workload(2, 1, 1, k, B, 64, [1000, 1000])
+    pair = Pair(w)
+    try:
+        for step in range(6):
+            base = (step % 2) * 500
+            sel = np.stack([np.arange(base + 7 * r, base + 7 * r + k) for r in range(2)])
+            _, h, m = pair.resolve_and_compare(0, sel)
+            assert m.tolist() == [k, k] and h.tolist() == [0, 0]
+            pair.compare_state(0)
+        pair.finish()
+    finally:
+        pair.close()
+
+
+def test_history_capacity_status():
+    w = tiny_workload(2, 1, 1, 2, 4, 16, [5, 6], steps=1)     # capacity = len + 2
+    pair = Pair(w)
+    try:
+        kv = torch.zeros((2, 1, 16), dtype=torch.uint8, device="cuda")
+        for _ in range(2):
+            pair.gpu.append(kv)
+        assert pair.gpu.status() == 0
+        pair.gpu.append(kv)
+        assert pair.gpu.status() == hs.STATUS_CAPACITY
+        st = pair.gpu.dump_state(0, 0)
+        assert st["len"] == 7 and st["newest"] == -1
+    finally:
+        pair.close()
+
+
+# ------------------------------------------------------------------ DSA / NSA / Quest shaped traces
+
+def test_c1_tiny_dsa_full():
+    w = inputs.c1_tiny_dsa()
+    h, m = run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, pool_every=16)
+    assert h + m == w.steps * w.top_k
+
+
+@pytest.mark.parametrize("S", [1, 2, 4, 8])
+def test_c2_shape_reduced_all_cluster_sizes(S):
+    # real k and B (several 1024-thread tiles), fewer requests / layers / tokens
+    w = inputs.c2_dsa_decode(num_requests=5, num_layers=2, steps=6, context=6000)
+    run_trace(w, w.steps, ctas_per_request=S, flags=hs.FLAG_DEBUG_VALIDATE)
+
+
+def test_ragged_sizes():
+    # k and B that are no multiples of the block size or of 32
+    w = inputs.Workload("ragged", inputs.KIND_DSA_MIX, 3, 2, 1, 1000, 3001, 80, [5000, 7000, 2500], 8,
+                        keep=800, recent_window=300, seed=3, config_id=9)
+    run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, pool_every=4)
+
+
+def test_maximum_sizes():
+    w = inputs.Workload("max", inputs.KIND_DSA_MIX, 2, 1, 1, hs.MAX_TOP_K, hs.MAX_CACHE_SLOTS, 16,
+                        [40000, 20000], 4, keep=3000, recent_window=2048, seed=4, config_id=10)
+    run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE)
+
+
+@pytest.mark.parametrize("overlap", [0.5, 0.98])
+def test_c3_shape_reduced_with_prefetch(overlap):
+    w = inputs.c3_dsa_long(overlap, steps=5, short_ctx=8192, long_ctx=65536, num_short=3)
+    run_trace(w, w.steps, use_prefetch=True, flags=hs.FLAG_DEBUG_VALIDATE)
+
+
+def test_c4_nsa_blocks_reduced():
+    w = inputs.c4_nsa_blocks(num_requests=4, num_layers=2, steps=70)
+    w.entry_bytes = 16384            # same block-granular selection, smaller blocks
+    run_trace(w, w.steps, pool_every=32)
+
+
+def test_c5_quest_pages_reduced():
+    w = inputs.c5_quest_pages(num_requests=3, num_layers=2, steps=20)
+    w.entry_bytes = 4096
+    run_trace(w, w.steps, pool_every=10)
+
+
+def test_skip_io_keeps_metadata_exact():
+    w = inputs.c2_dsa_decode(num_requests=2, num_layers=1, steps=4, context=5000)
+    pair = Pair(w, flags=hs.FLAG_SKIP_IO, oracle_bytes=False)
+    tr = inputs.Trace(w)
+    try:
+        for _ in range(4):
+            sel, app, _ = tr.step()
+            if app:
+                pair.append()
+            tab, _, _ = pair.resolve_and_compare(0, sel[0], check_bytes=False)
+            pair.compare_state(0)
+        # no record was fetched: every LRU slot still holds the zeros it was created with
+        tab_d = torch.from_numpy(tab).cuda()
+        got = pair.gpu.gather(0, tab_d).cpu().numpy()
+        lru = (tab % (w.cache_slots + 1)) != w.cache_slots
+        assert not got[lru].any()
+    finally:
+        tr.close()
+        pair.close()
+
+
+# ------------------------------------------------------------------ CUDA graph replay of whole steps
+
+def test_graph_replay_matches_oracle():
+    w = inputs.c3_dsa_long(0.75, steps=6, short_ctx=4096, long_ctx=16384, num_short=2)
+    pair = Pair(w)
+    tr = inputs.Trace(w)
+    dev = pair.dev
+    N, k, L, G, lpg = w.num_requests, w.top_k, w.num_layers, w.num_groups, w.layers_per_group
+    sel_d = torch.empty((G, N, k), dtype=torch.int32, device=dev)
+    kv_d = torch.empty((N, L, w.entry_bytes), dtype=torch.uint8, device=dev)
+    tabs = torch.empty((L, N, k), dtype=torch.int32, device=dev)
+    hits = torch.empty((L, N), dtype=torch.int32, device=dev)
+    misses = torch.empty((L, N), dtype=torch.int32, device=dev)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    try:
+        torch.cuda.synchronize()
+        with torch.cuda.stream(main):
+            graph.capture_begin()
+            pair.gpu.append(kv_d, stream=main)
+            for layer in range(L):
+                pair.gpu.resolve(layer, sel_d[layer // lpg], tabs[layer], hits[layer], misses[layer], stream=main)
+                if layer % lpg == 0:
+                    for l in range(layer + 1, layer + lpg):
+                        pair.gpu.prefetch(l, side)
+            graph.capture_end()
+        for step in range(w.steps):
+            sel, app, lens = tr.step()
+            assert app
+            kv = inputs.new_kv(w, lens - 1)
+            pair.oracle.append(kv)
+            kv_d.copy_(torch.from_numpy(kv))
+            sel_d.copy_(torch.from_numpy(sel))
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            for layer in range(L):
+                tab_o, h_o, m_o = pair.oracle.resolve(layer, sel[layer // lpg])
+                assert np.array_equal(tabs[layer].cpu().numpy(), tab_o)
+                assert np.array_equal(hits[layer].cpu().numpy(), h_o)
+                assert np.array_equal(misses[layer].cpu().numpy(), m_o)
+                pair.gpu.gather_check(layer, sel_d[layer // lpg], tabs[layer], pair.mism)
+                pair.compare_state(layer)
+            if step % 3 == 0:
+                for layer in range(L):
+                    pair.compare_whole_pool(layer)
+        pair.finish()
+    finally:
+        tr.close()
+        pair.close()
+
+
+# ------------------------------------------------------------------ boundary errors
+
+def test_create_rejects_bad_arguments():
+    hist = HostHistory(1, 64, 32)
+    try:
+        def make(**kw):
+            a = dict(num_requests=1, num_layers=1, layers_per_group=1, cache_slots=8, top_k=4, entry_bytes=32,
+                     capacity=[64], init_len=[10], host_history=[hist])
+            a.update(kw)
+            return HiSparse(**a)
+        for bad in (dict(top_k=9), dict(entry_bytes=40), dict(cache_slots=hs.MAX_CACHE_SLOTS + 1),
+                    dict(num_layers=3, layers_per_group=2), dict(init_len=[65]), dict(ctas_per_request=3)):
+            with pytest.raises(HiSparseError) as e:
+                make(**bad)
+            assert e.value.code == hs.EINVAL
+        pageable = np.zeros(64 * 32, dtype=np.uint8)
+        with pytest.raises(HiSparseError) as e:
+            make(host_history=[pageable.ctypes.data])
+        assert e.value.code == hs.ENOTPINNED
+        h = make()
+        sel = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+        with pytest.raises(HiSparseError) as e:
+            h.resolve(1, sel)
+        assert e.value.code == hs.EINVAL
+        with pytest.raises(HiSparseError):
+            h.prefetch(0, torch.cuda.Stream())
+        h.close()
+        kv, meta = hs.device_bytes(1, 1, 1, 8, 4, 32, [64])
+        assert kv == 1 * 1 * 9 * 32 and meta > 0
+    finally:
+        hist.free()
