@@ -68,6 +68,9 @@ struct DevState {
   int32_t *n_appends;
   uint32_t *ticket;
   uint32_t *status;
+  int meta_smem;                   // bytes of shared memory the metadata arrays take (ring follows)
+  int io_threads, io_depth, io_chunk;  // fetch pipeline: issuing threads, ring slots per thread, bytes per piece
+  unsigned long long *phase_ns;    // [N][16]: 8 globaltimer stamps, then 8 SM cycle-counter stamps (PHASE_TIMERS)
 };
 
 // ------------------------------------------------------------------------------------------ device helpers
@@ -80,33 +83,9 @@ __device__ __forceinline__ uint4 ld_host16(const void *p) {
   return v;
 }
 
-__device__ __forceinline__ void cluster_barrier() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
 // Multiplicative hash of a position into a table of H = 2^(32 - shift) entries.
 __device__ __forceinline__ uint32_t hash_pos(int32_t p, int shift) {
   return ((uint32_t)p * 0x9E3779B1u) >> shift;
-}
-
-// Block-wide exclusive prefix count of one flag per thread.  s_warp: 32 ints of scratch.
-__device__ __forceinline__ int block_flag_scan(bool flag, int *s_warp, int &total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-  const unsigned b = __ballot_sync(0xffffffffu, flag);
-  const int within = __popc(b & ((1u << lane) - 1u));
-  if (lane == 0) s_warp[warp] = __popc(b);
-  __syncthreads();
-  const int v = lane < nw ? s_warp[lane] : 0;
-  int incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += n;
-  }
-  const int warp_excl = __shfl_sync(0xffffffffu, incl - v, warp);
-  total = __shfl_sync(0xffffffffu, incl, 31);
-  __syncthreads();
-  return warp_excl + within;
 }
 
 __device__ __forceinline__ void history_state(const DevState &d, int r, int64_t &len, int64_t &newest) {
@@ -116,37 +95,379 @@ __device__ __forceinline__ void history_state(const DevState &d, int r, int64_t 
   newest = (na > 0 && il + na <= cap) ? il + na - 1 : -1;
 }
 
-// Phase 4 (Sec. 3.4): copy m records host -> cache for request r of `layer`.  The plan (position, slot) is read
-// from shared memory.  The work is flattened into 16-byte units so that consecutive threads read consecutive
-// host addresses across record boundaries; `part` of `nparts` blocks share it.
-__device__ __forceinline__ void fetch_records(const DevState &d, int r, int layer, int m, const int32_t *s_pos,
-                                              const int32_t *s_slot, int part, int nparts) {
-  const uint32_t upe = d.upe;
-  const uint8_t *hbase = d.host[r] + (int64_t)layer * d.cap[r] * d.E;
-  uint8_t *pbase = d.pool + (int64_t)layer * d.layer_pool_bytes + (int64_t)r * (d.B + 1) * d.E;
-  const uint64_t total = (uint64_t)m * upe;
-  const uint64_t stride = (uint64_t)nparts * blockDim.x;
-  for (uint64_t base = (uint64_t)part * blockDim.x + threadIdx.x; base < total; base += stride * kFetchUnroll) {
-    uint4 v[kFetchUnroll];
-    uint8_t *dst[kFetchUnroll];
-#pragma unroll
-    for (int i = 0; i < kFetchUnroll; ++i) {
-      const uint64_t u = base + (uint64_t)i * stride;
-      dst[i] = nullptr;
-      if (u < total) {
-        const uint32_t rec = (uint32_t)(u / upe);
-        const uint32_t off = (uint32_t)(u - (uint64_t)rec * upe);
-        v[i] = ld_host16(hbase + ((int64_t)s_pos[rec] * upe + off) * 16);
-        dst[i] = pbase + ((int64_t)s_slot[rec] * upe + off) * 16;
-      }
+// ---- Phase 4 (Sec. 3.4): fetch of the missing records as a bulk-async-copy (TMA) pipeline ----
+//
+// Records travel host -> shared memory -> cache slot with cp.async.bulk in both directions, so no thread holds
+// data in registers and a block keeps its whole staging ring (up to ~150 KB) in flight over the host link.
+// A record is cut into pieces of d.io_chunk bytes.  Each of the first d.io_threads threads of a block owns
+// d.io_depth ring slots and one mbarrier: it issues a batch of loads (one expect_tx for the batch), goes on with
+// other work, later waits for the batch, issues the stores to the cache slots and reuses its ring slots.  Threads
+// never wait for one another.  Every wait is bounded (2 s of %globaltimer); on expiry STATUS_TIMEOUT is set and
+// the thread stops fetching.
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  uint32_t done = 0;
+  uint64_t t0 = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    if ((spin & 63u) == 63u) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 2000000000ull) return false;
     }
-#pragma unroll
-    for (int i = 0; i < kFetchUnroll; ++i)
-      if (dst[i]) *reinterpret_cast<uint4 *>(dst[i]) = v[i];
   }
 }
 
+struct TmaFetch {
+  const uint8_t *hbase;
+  uint8_t *pbase;
+  const int32_t *s_pos, *s_slot;
+  uint32_t ring, bar;      // shared-memory addresses of this thread's ring slots and mbarrier
+  int64_t E, total;        // record bytes, number of pieces to move in this request
+  int chunk, ppr, depth, io_threads, part, nparts;
+  int batch;
+  uint32_t parity;
+  bool active;
+
+  __device__ __forceinline__ void init(const DevState &d, int r, int layer, int m, const int32_t *pos,
+                                       const int32_t *slot, unsigned char *ring_base, unsigned long long *bars,
+                                       int part_, int nparts_) {
+    const int tid = threadIdx.x;
+    E = d.E; chunk = d.io_chunk; depth = d.io_depth; io_threads = d.io_threads;
+    ppr = (int)((E + chunk - 1) / chunk);
+    total = (int64_t)m * ppr;
+    part = part_; nparts = nparts_;
+    s_pos = pos; s_slot = slot;
+    hbase = d.host[r] + (int64_t)layer * d.cap[r] * d.E;
+    pbase = d.pool + (int64_t)layer * d.layer_pool_bytes + (int64_t)r * (d.B + 1) * d.E;
+    ring = smem_u32(ring_base) + (uint32_t)tid * (uint32_t)(depth * chunk);
+    bar = smem_u32(bars + tid);
+    batch = 0; parity = 0;
+    active = tid < io_threads && m > 0 && !(d.flags & HISPARSE_FLAG_SKIP_IO);
+  }
+
+  // piece number of this thread's q-th transfer
+  __device__ __forceinline__ int64_t piece_of(int q) const {
+    return ((int64_t)q * io_threads + threadIdx.x) * nparts + part;
+  }
+
+  // Issues the loads of the next batch; false when this thread has nothing left.
+  __device__ __forceinline__ bool issue() {
+    if (!active) return false;
+    uint32_t bytes_total = 0;
+    for (int s = 0; s < depth; ++s) {
+      const int64_t c = piece_of(batch * depth + s);
+      if (c >= total) break;
+      const int piece = (int)(c % ppr);
+      const int64_t rest = E - (int64_t)piece * chunk;
+      bytes_total += (uint32_t)(rest < chunk ? rest : chunk);
+    }
+    if (bytes_total == 0) { active = false; return false; }
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes_total) : "memory");
+    for (int s = 0; s < depth; ++s) {
+      const int64_t c = piece_of(batch * depth + s);
+      if (c >= total) break;
+      const int64_t rec = c / ppr;
+      const int piece = (int)(c - rec * ppr);
+      const int64_t rest = E - (int64_t)piece * chunk;
+      const uint32_t bytes = (uint32_t)(rest < chunk ? rest : chunk);
+      const uint8_t *src = hbase + (int64_t)s_pos[rec] * E + (int64_t)piece * chunk;
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(ring + (uint32_t)(s * chunk)), "l"(src), "r"(bytes), "r"(bar) : "memory");
+    }
+    return true;
+  }
+
+  // Waits for the batch issued last, stores it to the cache slots and frees the ring slots.
+  __device__ __forceinline__ void complete(uint32_t *status) {
+    if (!mbar_wait_bounded(bar, parity)) {
+      atomicOr(status, HISPARSE_STATUS_TIMEOUT);
+      active = false;
+      return;
+    }
+    parity ^= 1u;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int s = 0; s < depth; ++s) {
+      const int64_t c = piece_of(batch * depth + s);
+      if (c >= total) break;
+      const int64_t rec = c / ppr;
+      const int piece = (int)(c - rec * ppr);
+      const int64_t rest = E - (int64_t)piece * chunk;
+      const uint32_t bytes = (uint32_t)(rest < chunk ? rest : chunk);
+      uint8_t *dst = pbase + (int64_t)s_slot[rec] * E + (int64_t)piece * chunk;
+      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                   ::"l"(dst), "r"(ring + (uint32_t)(s * chunk)), "r"(bytes) : "memory");
+    }
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // ring slots reusable
+    ++batch;
+  }
+
+  __device__ __forceinline__ void drain(uint32_t *status) {
+    bool pending = active;  // a batch is in flight whenever the thread is still active here
+    while (pending) {
+      complete(status);
+      pending = issue();
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+};
+
+__device__ __forceinline__ void fetch_barriers_init(unsigned long long *bars, int io_threads) {
+  if ((int)threadIdx.x < io_threads)
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + threadIdx.x)) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
 // ------------------------------------------------------------------------------------------ Resolve (Sec. 3.4)
+
+// Block-wide exclusive prefix sum of one int per thread (two barriers).  s_warp: 32 ints of scratch.
+__device__ __forceinline__ int block_scan_excl(int v, int *s_warp, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  const int w = lane < nw ? s_warp[lane] : 0;
+  int wincl = w;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, wincl, o);
+    if (lane >= o) wincl += n;
+  }
+  const int warp_excl = __shfl_sync(0xffffffffu, wincl - w, warp);
+  total = __shfl_sync(0xffffffffu, wincl, 31);
+  __syncthreads();
+  return warp_excl + incl - v;
+}
+
+// Asynchronous global -> shared staging (cp.async, 16 bytes per thread and step); falls back to plain 4- or
+// 2-byte copies when the size or an address is not a multiple of 16.  Complete after cp.async.wait_all + barrier.
+__device__ __forceinline__ void stage_async(void *smem_dst, const void *gmem_src, int bytes) {
+  const uint32_t sdst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  if (((bytes | (int)sdst | (int)(uintptr_t)gmem_src) & 15) == 0) {
+    for (int o = threadIdx.x * 16; o < bytes; o += blockDim.x * 16)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sdst + o), "l"((const char *)gmem_src + o) : "memory");
+  } else if (((bytes | (int)sdst | (int)(uintptr_t)gmem_src) & 3) == 0) {
+    for (int o = threadIdx.x * 4; o < bytes; o += blockDim.x * 4)
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + o), "l"((const char *)gmem_src + o) : "memory");
+  } else {
+    for (int o = threadIdx.x * 2; o < bytes; o += blockDim.x * 2)
+      *reinterpret_cast<uint16_t *>((char *)smem_dst + o) = *reinterpret_cast<const uint16_t *>((const char *)gmem_src + o);
+  }
+}
+
+// The selected set as an open-addressing hash table in shared memory (Phase 1): one 8-byte entry per bucket,
+// (position << 32) | row index, all ones = empty.  Key and value travel in one load, and several independent
+// probe sequences per thread are advanced together so that their shared-memory latencies overlap.
+constexpr unsigned long long kEmptyEntry = ~0ull;
+constexpr int kSelPerThread = HISPARSE_MAX_TOP_K / kThreads;  // row entries per thread
+
+template <int N>
+__device__ __forceinline__ void table_lookup(const unsigned long long *tab, const uint32_t mask, const int shift,
+                                             const int32_t (&key)[N], int32_t (&found)[N]) {
+  uint32_t h[N];
+  uint32_t open = 0;
+#pragma unroll
+  for (int i = 0; i < N; ++i) {
+    found[i] = -1;
+    h[i] = hash_pos(key[i], shift);
+    if (key[i] >= 0) open |= 1u << i;
+  }
+  for (uint32_t round = 0; open && round <= mask; ++round) {
+    unsigned long long e[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+      if ((open >> i) & 1u) e[i] = tab[h[i]];
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+      if ((open >> i) & 1u) {
+        if ((int32_t)(e[i] >> 32) == key[i]) {
+          found[i] = (int32_t)(uint32_t)e[i];
+          open &= ~(1u << i);
+        } else if (e[i] == kEmptyEntry) {
+          open &= ~(1u << i);
+        } else {
+          h[i] = (h[i] + 1u) & mask;
+        }
+      }
+  }
+}
+
+// Everything the first block of a cluster does before the fetch can start: Phases 1-3 of Sec. 3.4.
+// IPT = entries of the recency order per thread (B <= IPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
+// the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
+// the untouched slots compacted at its front, and s_hitbits / s_vicbits the per-slot marks.
+template <int IPT>
+__device__ __forceinline__ void resolve_metadata(const DevState &d, const int r, const int64_t rg, const int32_t *row,
+                                                 int32_t *s_sel, int32_t *s_out, int32_t *s_plan_pos,
+                                                 int32_t *s_plan_slot, unsigned long long *s_tab, uint32_t *s_hitbits,
+                                                 uint32_t *s_vicbits, uint16_t *s_order, int *s_warp, int *s_misc,
+                                                 const uint32_t hit_stamp, unsigned long long *stamps, int &m,
+                                                 int &n_nonhit, uint32_t &my_status) {
+  constexpr int T = kThreads;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int k = d.k, B = d.B, H = d.H, W = d.W;
+  const uint32_t mask = (uint32_t)(H - 1);
+  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+  uint32_t *last_use = d.last_use + rg * B;
+
+  // Phase 1: stage the row and the recency order (one round trip to HBM), clear the marks and the table.
+  stage_async(s_sel, row, k * 4);
+  stage_async(s_order, d.order + rg * B, B * 2);
+  int64_t len, newest;
+  history_state(d, r, len, newest);
+  const int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)(rg - (int64_t)r * d.G) * d.cap[r];
+  for (int i = tid; i < H; i += T) s_tab[i] = kEmptyEntry;
+  for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
+  if (tid < 4) s_misc[tid] = 0;
+  if (timers && tid == 0) stamps[8] = clock64();
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  if (timers && tid == 0) stamps[9] = clock64();
+
+  // Phase 2: hit detection through the page table (position -> slot): all of a thread's lookups are issued
+  // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
+  // resident go into the hash table (position -> row index), whose only job is to catch a position that is
+  // selected twice, so that it claims one victim, not two.
+  int32_t pos[kSelPerThread], got[kSelPerThread];
+#pragma unroll
+  for (int i = 0; i < kSelPerThread; ++i) {
+    const int j = tid + i * T;
+    pos[i] = j < k ? s_sel[j] : -1;
+    const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
+    if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
+    if (!ok) pos[i] = -1;
+    got[i] = ok ? __ldg(p2s + pos[i]) : -1;
+  }
+  int my_valid = 0;
+#pragma unroll
+  for (int i = 0; i < kSelPerThread; ++i) {
+    const int j = tid + i * T;
+    if (j >= k) break;
+    const int32_t p = pos[i];
+    int32_t o = -1;
+    if (p >= 0) {
+      if ((int64_t)p == newest) {  // reserved newest-record slot, outside the LRU set
+        o = B;
+        if (atomicExch(&s_misc[2], 1) == 0) ++my_valid; else my_status |= HISPARSE_STATUS_DUPLICATE;
+      } else if (got[i] >= 0) {
+        const int s = got[i];
+        o = s;
+        const uint32_t bit = 1u << (s & 31);
+        if (atomicOr(&s_hitbits[s >> 5], bit) & bit) {
+          my_status |= HISPARSE_STATUS_DUPLICATE;  // the same resident position again: same slot, counted once
+        } else {
+          ++my_valid;
+          last_use[s] = hit_stamp;
+        }
+      } else {
+        o = kMiss;
+        ++my_valid;
+        const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)j;
+        uint32_t h = hash_pos(p, d.hshift);
+        for (uint32_t it = 0; it <= mask; ++it) {
+          const unsigned long long old = atomicCAS(&s_tab[h], kEmptyEntry, entry);
+          if (old == kEmptyEntry) break;
+          if ((int32_t)(old >> 32) == p) {  // selected twice: the lowest row index owns the entry
+            atomicMin(&s_tab[h], entry);
+            s_misc[0] = 1;
+            break;
+          }
+          h = (h + 1u) & mask;
+        }
+      }
+    }
+    s_out[j] = o;
+  }
+  __syncthreads();
+  if (timers && tid == 0) stamps[10] = clock64();
+  if (s_misc[0]) {  // rare: every later occurrence of a repeated missing position follows the first one
+    for (int j = tid; j < k; j += T) {
+      if (s_out[j] == kMiss) {
+        const int32_t key[1] = {s_sel[j]};
+        int32_t owner[1];
+        table_lookup<1>(s_tab, mask, d.hshift, key, owner);
+        if (owner[0] != j) {
+          s_out[j] = kDupBase - owner[0];
+          --my_valid;
+          my_status |= HISPARSE_STATUS_DUPLICATE;
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) my_valid += __shfl_xor_sync(0xffffffffu, my_valid, o);
+  if (lane == 0 && my_valid) atomicAdd(&s_misc[1], my_valid);
+  if (timers && tid == 0) { stamps[1] = global_ns(); stamps[11] = clock64(); }
+  __syncthreads();
+  if (timers && tid == 0) { stamps[2] = global_ns(); stamps[12] = clock64(); }
+
+  // Phase 3: ONE block scan over packed counts (non-hit slots in recency order | misses in selection order).
+  // Thread t owns IPT consecutive entries of the recency order and kSelPerThread consecutive row entries.
+  {
+    int slot[IPT];
+    uint32_t nh_mask = 0, miss_mask = 0;
+#pragma unroll
+    for (int i = 0; i < IPT; ++i) {
+      const int q = tid * IPT + i;
+      slot[i] = 0;
+      if (q < B) {
+        slot[i] = s_order[q];
+        if (!((s_hitbits[slot[i] >> 5] >> (slot[i] & 31)) & 1u)) nh_mask |= 1u << i;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i) {
+      const int j = tid * kSelPerThread + i;
+      if (j < k && s_out[j] == kMiss) miss_mask |= 1u << i;
+    }
+    int total;
+    const int excl = block_scan_excl((__popc(nh_mask) << 16) | __popc(miss_mask), s_warp, total);
+    m = total & 0xffff;
+    n_nonhit = total >> 16;
+    int mrank = excl & 0xffff, nrank = excl >> 16;
+    // the i-th miss (selection order) takes the i-th non-hit slot of the recency order
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+      if ((miss_mask >> i) & 1u) s_plan_pos[mrank++] = tid * kSelPerThread + i;
+#pragma unroll
+    for (int i = 0; i < IPT; ++i)
+      if ((nh_mask >> i) & 1u) {
+        const int s = slot[i];
+        if (nrank < m) {
+          s_plan_slot[nrank] = s;
+          atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
+        } else {
+          s_order[nrank - m] = (uint16_t)s;  // in place: every thread read its entries before the scan's barriers
+        }
+        ++nrank;
+      }
+  }
+  if (timers && tid == 0) stamps[13] = clock64();
+  __syncthreads();
+  for (int i = tid; i < m; i += T) {
+    const int j = s_plan_pos[i];
+    s_out[j] = s_plan_slot[i];
+    s_plan_pos[i] = s_sel[j];
+  }
+  __syncthreads();
+  if (timers && tid == 0) stamps[14] = clock64();
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ sel, int32_t *__restrict__ table,
@@ -154,158 +475,77 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_warp[32];
   __shared__ int s_misc[4];  // [0] any duplicate  [1] valid distinct selections
-  const int tid = threadIdx.x, T = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int T = kThreads;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x / S, part = blockIdx.x - r * S;
   const int g = layer / d.lpg;
   const int k = d.k, B = d.B, H = d.H, W = d.W;
   const int64_t rg = (int64_t)r * d.G + g;
+  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+  unsigned long long *stamps = d.phase_ns + (int64_t)r * 16;
 
-  int32_t *s_sel = reinterpret_cast<int32_t *>(smem_raw);
+  unsigned long long *s_tab = reinterpret_cast<unsigned long long *>(smem_raw);
+  int32_t *s_sel = reinterpret_cast<int32_t *>(s_tab + H);
   int32_t *s_out = s_sel + k;
-  int32_t *s_plan_pos = s_out + k;   // first the row indices of the misses, then their positions
+  int32_t *s_plan_pos = s_out + k;        // first the row indices of the misses, then their positions
   int32_t *s_plan_slot = s_plan_pos + k;  // victims, in order
-  uint32_t *s_tab = reinterpret_cast<uint32_t *>(s_plan_slot + k);
-  uint32_t *s_hitbits = s_tab + H;
+  uint32_t *s_hitbits = reinterpret_cast<uint32_t *>(s_plan_slot + k);
   uint32_t *s_vicbits = s_hitbits + W;
   int32_t *s_hitpre = reinterpret_cast<int32_t *>(s_vicbits + W);
   int32_t *s_vicpre = s_hitpre + W;
   uint16_t *s_order = reinterpret_cast<uint16_t *>(s_vicpre + W);
+  unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
+  unsigned char *s_ring = smem_raw + d.meta_smem + kThreads * 8;
 
-  int m = 0;
+  fetch_barriers_init(s_bars, d.io_threads);  // made visible by the barriers below, long before first use
+  TmaFetch fetch;
+  int m = 0, n_nonhit = 0;
+  uint32_t t = 0;
   if (part == 0) {
-    int64_t len, newest;
-    history_state(d, r, len, newest);
-    const uint32_t t = d.t[rg] + 1u;
+    if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
+    t = d.t[rg] + 1u;
     const uint32_t hit_stamp = 2u * t + 1u, miss_stamp = 2u * t;
+    uint32_t my_status = 0;
+    const int32_t *row = sel + (int64_t)r * k;
+#define HS_META(IPT)                                                                                              \
+  resolve_metadata<IPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits, s_order, \
+                        s_warp, s_misc, hit_stamp, stamps, m, n_nonhit, my_status)
+    if (B <= 4 * T) HS_META(4);
+    else if (B <= 8 * T) HS_META(8);
+    else HS_META(16);
+#undef HS_META
+    if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
+    // Phase 4 starts here: the first batch of host loads is in flight while the metadata is written back
+    fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
+    fetch.issue();
+    // Phase 5, metadata half: page table, slot array, stamps, plan
     int32_t *slot_pos = d.slot_pos + rg * B;
     uint32_t *last_use = d.last_use + rg * B;
-    uint16_t *order = d.order + rg * B;
     int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
-    const int32_t *row = sel + (int64_t)r * k;
+    int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
+    for (int i = tid; i < m; i += T) {
+      const int v = s_plan_slot[i];
+      const int32_t p = s_plan_pos[i];
+      const int32_t old = slot_pos[v];
+      if (old >= 0) p2s[old] = -1;
+      slot_pos[v] = p;
+      p2s[p] = v;
+      last_use[v] = miss_stamp;
+      plan_pos_g[i] = p;
+      plan_slot_g[i] = v;
+    }
+    if (tid == 0) d.plan_n[rg] = m;
+    if (my_status) atomicOr(d.status, my_status);
+    if (S > 1) {
+      __threadfence();
+      __syncthreads();
+    }
+  }
+  // The plan is public: the other blocks of the cluster start fetching while this one publishes.
+  if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
-    // Phase 1: stage the selected positions and hash them (value = row index + 1, 0 = empty).
-    for (int i = tid; i < H; i += T) s_tab[i] = 0u;
-    for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
-    if (tid < 4) s_misc[tid] = 0;
-    for (int j = tid; j < k; j += T) s_sel[j] = row[j];
-    __syncthreads();
-
-    uint32_t my_status = 0;
-    int my_valid = 0;
-    for (int j = tid; j < k; j += T) {
-      const int32_t p = s_sel[j];
-      int32_t o = -1;
-      if (p == -1) {
-      } else if (p < 0 || (int64_t)p >= len) {
-        my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
-      } else {
-        o = (int64_t)p == newest ? B : kMiss;
-        ++my_valid;
-        uint32_t hsh = hash_pos(p, d.hshift);
-        for (int it = 0; it < H; ++it) {
-          uint32_t cur = *(volatile uint32_t *)&s_tab[hsh];
-          if (cur == 0u) {
-            cur = atomicCAS(&s_tab[hsh], 0u, (uint32_t)j + 1u);
-            if (cur == 0u) break;
-          }
-          if (s_sel[cur - 1u] == p) {  // the same position again: the lowest row index owns the entry
-            atomicMin(&s_tab[hsh], (uint32_t)j + 1u);
-            s_misc[0] = 1;
-            break;
-          }
-          hsh = (hsh + 1u) & (uint32_t)(H - 1);
-        }
-      }
-      s_out[j] = o;
-    }
-    __syncthreads();
-    if (s_misc[0]) {  // rare: mark every later occurrence of a repeated position
-      for (int j = tid; j < k; j += T) {
-        if (s_out[j] == kMiss || s_out[j] == B) {
-          const int32_t p = s_sel[j];
-          uint32_t hsh = hash_pos(p, d.hshift);
-          for (int it = 0; it < H; ++it) {
-            const uint32_t cur = s_tab[hsh];
-            if (cur == 0u) break;
-            if (s_sel[cur - 1u] == p) {
-              if ((int)cur - 1 != j) {
-                s_out[j] = kDupBase - ((int)cur - 1);
-                --my_valid;
-                my_status |= HISPARSE_STATUS_DUPLICATE;
-              }
-              break;
-            }
-            hsh = (hsh + 1u) & (uint32_t)(H - 1);
-          }
-        }
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) my_valid += __shfl_xor_sync(0xffffffffu, my_valid, o);
-    if (lane == 0 && my_valid) atomicAdd(&s_misc[1], my_valid);
-    __syncthreads();
-
-    // Phase 2: probe the position held by every slot; hits keep their slot and are stamped first.
-    for (int base = 0; base < B; base += T) {
-      const int s = base + tid;
-      bool hit = false;
-      if (s < B) {
-        const int32_t p = slot_pos[s];
-        if (p >= 0) {
-          uint32_t hsh = hash_pos(p, d.hshift);
-          for (int it = 0; it < H; ++it) {
-            const uint32_t cur = s_tab[hsh];
-            if (cur == 0u) break;
-            if (s_sel[cur - 1u] == p) {
-              if (s_out[cur - 1u] == kMiss) {
-                s_out[cur - 1u] = s;
-                hit = true;
-                last_use[s] = hit_stamp;
-              }
-              break;
-            }
-            hsh = (hsh + 1u) & (uint32_t)(H - 1);
-          }
-        }
-      }
-      const unsigned bal = __ballot_sync(0xffffffffu, hit);
-      if (lane == 0 && base + warp * 32 < B) s_hitbits[(base >> 5) + warp] = bal;
-    }
-    __syncthreads();
-
-    // Phase 3a: compact the misses in selection order.
-    for (int base = 0; base < k; base += T) {
-      const int j = base + tid;
-      const bool flag = j < k && s_out[j] == kMiss;
-      int total;
-      const int rank = block_flag_scan(flag, s_warp, total);
-      if (flag) s_plan_pos[m + rank] = j;
-      m += total;
-    }
-    // Phase 3b: walk the recency order; the first m slots that were not hit are the victims, in order;
-    // the other non-hit slots keep their relative order at the front of the new order.
-    int n_nonhit = 0;
-    for (int base = 0; base < B; base += T) {
-      const int q = base + tid;
-      int s = 0;
-      bool flag = false;
-      if (q < B) {
-        s = order[q];
-        flag = !((s_hitbits[s >> 5] >> (s & 31)) & 1u);
-      }
-      int total;
-      const int rank = n_nonhit + block_flag_scan(flag, s_warp, total);
-      if (flag) {
-        if (rank < m) {
-          s_plan_slot[rank] = s;
-          atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
-        } else {
-          s_order[rank - m] = (uint16_t)s;
-        }
-      }
-      n_nonhit += total;
-    }
-    __syncthreads();
+  if (part == 0) {
+    uint16_t *order = d.order + rg * B;
     // new order = untouched ++ victims by slot ++ hits by slot: word-level prefix counts, then one pass.
     if (warp == 0) {
       int run_h = 0, run_v = 0;
@@ -323,6 +563,15 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
         run_v += __shfl_sync(0xffffffffu, iv, 31);
       }
     }
+    // Phase 5: the slot table in selection order (does not depend on the order rewrite)
+    int32_t *trow = table + (int64_t)r * k;
+    int32_t *arow = d.anchor_out + rg * k;
+    for (int j = tid; j < k; j += T) {
+      int32_t o = s_out[j];
+      if (o <= kDupBase) o = s_out[kDupBase - o];
+      trow[j] = o < 0 ? -1 : r * (B + 1) + o;
+      if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
+    }
     __syncthreads();
     const int n_surv = n_nonhit - m;
     for (int s = tid; s < B; s += T) {
@@ -332,57 +581,40 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       if (vw & bit) s_order[n_surv + s_vicpre[w] + __popc(vw & lt)] = (uint16_t)s;
       else if (hw & bit) s_order[n_nonhit + s_hitpre[w] + __popc(hw & lt)] = (uint16_t)s;
     }
-    // Phase 3c / 5: the i-th miss takes the i-th victim; page table, slot array, stamps, plan.
-    int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
-    for (int i = tid; i < m; i += T) {
-      const int j = s_plan_pos[i];
-      const int v = s_plan_slot[i];
-      const int32_t p = s_sel[j];
-      const int32_t old = slot_pos[v];
-      if (old >= 0) p2s[old] = -1;
-      slot_pos[v] = p;
-      p2s[p] = v;
-      last_use[v] = miss_stamp;
-      s_out[j] = v;
-      plan_pos_g[i] = p;
-      plan_slot_g[i] = v;
-      s_plan_pos[i] = p;
-    }
     __syncthreads();
-    // Phase 5: publish the slot table in selection order, the new recency order and the counters.
-    int32_t *trow = table + (int64_t)r * k;
-    int32_t *arow = d.anchor_out + rg * k;
-    for (int j = tid; j < k; j += T) {
-      int32_t o = s_out[j];
-      if (o <= kDupBase) o = s_out[kDupBase - o];
-      trow[j] = o < 0 ? -1 : r * (B + 1) + o;
-      if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
-    }
     for (int q = tid; q < B; q += T) order[q] = s_order[q];
     if (tid == 0) {
       const int nvalid = s_misc[1];
       hits_out[r] = nvalid - m;
       misses_out[r] = m;
-      d.plan_n[rg] = m;
       d.anchor_hits[rg] = nvalid - m;
       d.anchor_misses[rg] = m;
       d.t[rg] = t;
     }
-    if (my_status) atomicOr(d.status, my_status);
+    if (timers && tid == 0) stamps[4] = global_ns();
   }
 
   if (S > 1) {
-    __threadfence();
-    cluster_barrier();
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     if (part != 0) {
       m = __ldcg(d.plan_n + rg);
       const int32_t *pp = d.plan_pos + rg * k, *ps = d.plan_slot + rg * k;
       for (int i = tid; i < m; i += T) { s_plan_pos[i] = __ldcg(pp + i); s_plan_slot[i] = __ldcg(ps + i); }
       __syncthreads();
+      fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, part, S);
+      fetch.issue();
     }
   }
-  // Phase 4: fetch the missing records.
-  if (!(d.flags & HISPARSE_FLAG_SKIP_IO)) fetch_records(d, r, layer, m, s_plan_pos, s_plan_slot, part, S);
+  // Phase 4, rest: wait for the batches, store them into the cache slots, issue what is left.
+  fetch.drain(d.status);
+  if (timers) {
+    __syncthreads();
+    if (tid == 0) {
+      const unsigned long long now = global_ns();
+      if (part == 0) stamps[5] = now;
+      atomicMax(&stamps[6], now);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------ plan replay (Sec. 3.5)
@@ -392,13 +624,19 @@ __global__ void __launch_bounds__(kThreads, 1) replay_kernel(const DevState d, c
   extern __shared__ __align__(16) unsigned char smem_raw[];
   int32_t *s_plan_pos = reinterpret_cast<int32_t *>(smem_raw);
   int32_t *s_plan_slot = s_plan_pos + d.k;
+  unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
+  unsigned char *s_ring = smem_raw + d.meta_smem + kThreads * 8;
   const int r = blockIdx.x / S, part = blockIdx.x - r * S;
   const int64_t rg = (int64_t)r * d.G + layer / d.lpg;
   const int m = d.plan_n[rg];
   const int32_t *pp = d.plan_pos + rg * d.k, *ps = d.plan_slot + rg * d.k;
+  fetch_barriers_init(s_bars, d.io_threads);
   for (int i = threadIdx.x; i < m; i += blockDim.x) { s_plan_pos[i] = pp[i]; s_plan_slot[i] = ps[i]; }
   __syncthreads();
-  if (!(d.flags & HISPARSE_FLAG_SKIP_IO)) fetch_records(d, r, layer, m, s_plan_pos, s_plan_slot, part, S);
+  TmaFetch fetch;
+  fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, part, S);
+  fetch.issue();
+  fetch.drain(d.status);
 }
 
 // A shared layer reuses its anchor's slot table (same local slots, same request offsets) and counts.
@@ -638,7 +876,7 @@ int hash_size(int k) {
 
 size_t resolve_smem_bytes(int B, int k) {
   const int H = hash_size(k), W = (B + 31) / 32;
-  return (size_t)4 * k * 4 + (size_t)H * 4 + (size_t)4 * W * 4 + (size_t)B * 2;
+  return (size_t)H * 8 + (size_t)4 * k * 4 + (size_t)4 * W * 4 + (size_t)B * 2;
 }
 
 cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
@@ -741,11 +979,19 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   for (int r = 0; r < N; ++r) { h->p2s_off[r] = off; off += h->cap[r] * G; }
   h->p2s_total = off;
 
-  h->resolve_smem = resolve_smem_bytes(B, k);
-  h->replay_smem = (size_t)2 * k * 4;
   int max_optin = 0;
   if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
-  if (h->resolve_smem + 1024 > (size_t)max_optin) return fail(HISPARSE_EINVAL);
+  // shared memory: metadata arrays, one mbarrier per thread, then the staging ring of the fetch pipeline,
+  // which takes whatever is left (pieces of at most 8 KB; at least one piece must fit)
+  d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
+  const int64_t ring_room = (int64_t)max_optin - 1024 - d.meta_smem - kThreads * 8;
+  if (ring_room < 16) return fail(HISPARSE_EINVAL);
+  d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
+  const int slots = (int)(ring_room / d.io_chunk);
+  d.io_threads = std::min(slots, kThreads);
+  d.io_depth = std::min(slots / d.io_threads, 8);
+  h->resolve_smem = (size_t)d.meta_smem + kThreads * 8 + (size_t)d.io_threads * d.io_depth * d.io_chunk;
+  h->replay_smem = h->resolve_smem;   // same offsets, so that both kernels share the pipeline's geometry
   if (cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaFuncSetAttribute(replay_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
 
@@ -790,6 +1036,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRY(dev_alloc(h, &d.n_appends, 1));
   HS_TRY(dev_alloc(h, &d.ticket, 1));
   HS_TRY(dev_alloc(h, &d.status, 1));
+  HS_TRY(dev_alloc(h, &d.phase_ns, (size_t)N * 16));
 #undef HS_TRY
   d.cap = h->d_cap; d.init_len = h->d_init_len; d.p2s_off = h->d_p2s_off; d.host = h->d_host;
 
@@ -810,6 +1057,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRYC(cudaMemset(d.n_appends, 0, 4));
   HS_TRYC(cudaMemset(d.ticket, 0, 4));
   HS_TRYC(cudaMemset(d.status, 0, 4));
+  HS_TRYC(cudaMemset(d.phase_ns, 0, (size_t)N * 16 * 8));
   init_order_kernel<<<296, 256>>>(d.order, (int64_t)NG * B, B);
   HS_TRYC(cudaGetLastError());
 
@@ -1012,6 +1260,14 @@ int hisparse_dump_plan(hisparse_t *h, int req, int layer, int32_t *plan_pos, int
   HS_CUDA(cudaMemcpy(n, h->d.plan_n + rg, 4, cudaMemcpyDeviceToHost));
   if (plan_pos) HS_CUDA(cudaMemcpy(plan_pos, h->d.plan_pos + rg * h->d.k, (size_t)h->d.k * 4, cudaMemcpyDeviceToHost));
   if (plan_slot) HS_CUDA(cudaMemcpy(plan_slot, h->d.plan_slot + rg * h->d.k, (size_t)h->d.k * 4, cudaMemcpyDeviceToHost));
+  return HISPARSE_OK;
+}
+
+int hisparse_phase_times(hisparse_t *h, uint64_t *out) {
+  if (!h || !out) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  HS_CUDA(cudaMemcpy(out, h->d.phase_ns, (size_t)h->d.N * 16 * 8, cudaMemcpyDeviceToHost));
   return HISPARSE_OK;
 }
 

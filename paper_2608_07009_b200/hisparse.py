@@ -15,7 +15,7 @@ import numpy as np
 from . import build as _build
 
 OK, EINVAL, ENOTPINNED, ENOMEM, ECUDA, ESTATE = 0, -1, -2, -3, -4, -5
-FLAG_SKIP_IO, FLAG_DEBUG_VALIDATE, FLAG_INLINE_WRITE_THROUGH = 1, 2, 4
+FLAG_SKIP_IO, FLAG_DEBUG_VALIDATE, FLAG_INLINE_WRITE_THROUGH, FLAG_PHASE_TIMERS = 1, 2, 4, 8
 STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, STATUS_CAPACITY, STATUS_INCONSISTENT, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 MAX_CACHE_SLOTS, MAX_TOP_K = 16384, 4096
 
@@ -23,7 +23,7 @@ EXPORTS = [
     "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch",
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
     "hisparse_clear_status", "hisparse_dump_state", "hisparse_dump_plan", "hisparse_device_bytes",
-    "hisparse_launch_geometry", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
+    "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
     "hisparse_scatter_read_probe", "hisparse_strerror", "hisparse_last_cuda_error",
 ]
 
@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
             "hisparse_dump_plan": ([vp, i32, i32, vp, vp, P(ctypes.c_int32)], i32),
             "hisparse_device_bytes": ([P(Config), P(sz), P(sz)], i32),
             "hisparse_launch_geometry": ([vp, P(ctypes.c_int32), P(ctypes.c_int32), P(ctypes.c_int32)], i32),
+            "hisparse_phase_times": ([vp, vp], i32),
             "hisparse_host_alloc": ([sz, P(vp)], i32),
             "hisparse_host_free": ([vp], i32),
             "hisparse_host_link_probe": ([i32, sz, i32, P(ctypes.c_double)], i32),
@@ -269,6 +270,12 @@ class HiSparse:
         _check(lib().hisparse_dump_plan(self._h, req, layer, pos.ctypes.data, slot.ctypes.data, ctypes.byref(n)),
                "hisparse_dump_plan")
         return pos[: n.value].copy(), slot[: n.value].copy()
+
+    def phase_times(self) -> np.ndarray:
+        """uint64 [N][16] stamps of the last anchor resolve (needs FLAG_PHASE_TIMERS): 8 in ns, 8 in SM cycles."""
+        out = np.zeros((self.N, 16), dtype=np.uint64)
+        _check(lib().hisparse_phase_times(self._h, out.ctypes.data), "hisparse_phase_times")
+        return out
 
     def launch_geometry(self):
         s, t, m = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
