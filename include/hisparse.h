@@ -40,6 +40,7 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
 #define HISPARSE_ENOMEM (-3)      /* device or host allocation failed                                */
 #define HISPARSE_ECUDA (-4)       /* a CUDA call failed; hisparse_last_cuda_error() has the code      */
 #define HISPARSE_ESTATE (-5)      /* call not valid now (e.g. prefetch of a layer whose anchor has not run) */
+#define HISPARSE_ETOOBIG (-6)     /* geometry exceeds the fixed scratch of hisparse_resolve_noalloc          */
 
 /* create flags */
 #define HISPARSE_FLAG_SKIP_IO 1u          /* timing mode of Sec. 4.6's "no-IO oracle": misses are resolved
@@ -203,6 +204,62 @@ int hisparse_host_link_probe(int device, size_t bytes, int reps, double *gb_per_
  * as *gb_per_s.  Allocates and frees its own device buffers.  Synchronises. */
 int hisparse_scatter_read_probe(int device, const void *host_buf, size_t host_bytes, int64_t entry_bytes,
                                 int32_t num_records, int32_t num_ctas, int reps, double *gb_per_s);
+
+/*
+ * hisparse_resolve_noalloc — Resolve for callers that must not allocate device memory.  (The paper has no
+ * counterpart of this entry point; it exists for integration.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits — an engine that has handed all of
+ * HBM to its own pool allocator at start-up and forbids later driver allocations, a plugin called while the
+ * host application is capturing a stream (allocation calls are illegal during capture), or a latency-critical
+ * path that may not take the driver's allocation lock.  hisparse_create allocates its caches and metadata with
+ * cudaMalloc, so such callers cannot use a handle.  Here the caller owns ALL persistent state of one layer's
+ * caches and passes it in; the only memory the kernel needs beyond those inputs and outputs — its scratch: the
+ * miss plan that the blocks of a cluster hand to one another, and a few counters — lives in a fixed array that
+ * is part of the library image (about 0.5 MB of device memory on every GPU that loads the library, held until
+ * the process exits).  The call allocates nothing and frees nothing, neither directly nor through a library.
+ *
+ * Limits (HISPARSE_ETOOBIG beyond them): num_requests <= HISPARSE_NOALLOC_MAX_REQUESTS and
+ * num_requests * top_k <= HISPARSE_NOALLOC_MAX_SELECTIONS; otherwise the limits of hisparse_create apply
+ * (HISPARSE_EINVAL).  One layer per state struct, no shared-selection groups, no prefetch.
+ *
+ * The first call on a device looks up the device address of the scratch array and raises the kernel's
+ * shared-memory limit (with that device current); make that first call before any stream capture begins.
+ * Later calls only enqueue a memset of the scratch counters and the kernel on `stream`.
+ * Every call on a device shares the one scratch array, which keeps the previous call's contents: the call
+ * clears what has to start from zero itself, and two calls whose kernels overlap on the GPU (different streams)
+ * race on it — serialise them.
+ *
+ * Semantics are exactly those of hisparse_resolve on an anchor layer; the state arrays use the layouts listed
+ * below and must start as: slot_pos = -1, last_use = 0, lru_order[r][i] = i, pos2slot = -1, resolves = 0, pool
+ * arbitrary.  *status_dev (may be NULL) receives HISPARSE_STATUS_* bits by atomic OR; the caller clears it.
+ */
+#define HISPARSE_NOALLOC_MAX_REQUESTS 1024
+#define HISPARSE_NOALLOC_MAX_SELECTIONS 65536
+
+typedef struct {
+  int32_t num_requests;          /* N                                                                     */
+  int32_t cache_slots;           /* B                                                                     */
+  int32_t top_k;                 /* k                                                                     */
+  int64_t entry_bytes;           /* E, multiple of 16                                                     */
+  int32_t device;                /* CUDA device ordinal the pointers below belong to                      */
+  void *pool_dev;                /* uint8 [N][B+1][E]: this layer's cache pool (slot B = newest record)   */
+  int32_t *slot_pos_dev;         /* int32 [N][B]                                                          */
+  uint32_t *last_use_dev;        /* uint32 [N][B]                                                         */
+  uint16_t *lru_order_dev;       /* uint16 [N][B]                                                         */
+  int32_t *pos2slot_dev;         /* int32, request r's page table at [p2s_offset[r], p2s_offset[r] + capacity[r]) */
+  const int64_t *capacity_dev;   /* int64 [N]                                                             */
+  const int64_t *init_len_dev;   /* int64 [N]: history length before any append                           */
+  const int64_t *p2s_offset_dev; /* int64 [N]                                                             */
+  void *const *host_layer_dev;   /* [N] device-visible addresses of this layer's pinned host history,
+                                    each laid out [capacity[r]][E]                                        */
+  uint32_t *resolves_dev;        /* uint32 [N]: resolves done so far per request                          */
+  const int32_t *num_appends_dev;/* int32 scalar: records appended so far (length = init_len + appends)   */
+} hisparse_external_state_t;
+
+int hisparse_resolve_noalloc(const hisparse_external_state_t *state, const int32_t *sel_dev,
+                             int32_t *slot_table_dev, int32_t *hits_dev, int32_t *misses_dev,
+                             uint32_t *status_dev, void *stream);
 
 const char *hisparse_strerror(int code);
 int hisparse_last_cuda_error(void);

@@ -14,7 +14,8 @@ import numpy as np
 
 from . import build as _build
 
-OK, EINVAL, ENOTPINNED, ENOMEM, ECUDA, ESTATE = 0, -1, -2, -3, -4, -5
+OK, EINVAL, ENOTPINNED, ENOMEM, ECUDA, ESTATE, ETOOBIG = 0, -1, -2, -3, -4, -5, -6
+NOALLOC_MAX_REQUESTS, NOALLOC_MAX_SELECTIONS = 1024, 65536
 FLAG_SKIP_IO, FLAG_DEBUG_VALIDATE, FLAG_INLINE_WRITE_THROUGH, FLAG_PHASE_TIMERS = 1, 2, 4, 8
 STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, STATUS_CAPACITY, STATUS_INCONSISTENT, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 MAX_CACHE_SLOTS, MAX_TOP_K = 16384, 4096
@@ -24,7 +25,7 @@ EXPORTS = [
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
     "hisparse_clear_status", "hisparse_dump_state", "hisparse_dump_plan", "hisparse_device_bytes",
     "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
-    "hisparse_scatter_read_probe", "hisparse_strerror", "hisparse_last_cuda_error",
+    "hisparse_scatter_read_probe", "hisparse_resolve_noalloc", "hisparse_strerror", "hisparse_last_cuda_error",
 ]
 
 
@@ -43,6 +44,18 @@ class Config(ctypes.Structure):
         ("cache_slots", ctypes.c_int32), ("top_k", ctypes.c_int32), ("entry_bytes", ctypes.c_int64),
         ("capacity", ctypes.c_void_p), ("init_len", ctypes.c_void_p), ("host_history", ctypes.c_void_p),
         ("device", ctypes.c_int32), ("flags", ctypes.c_uint32), ("ctas_per_request", ctypes.c_int32),
+    ]
+
+
+class ExternalState(ctypes.Structure):
+    """hisparse_external_state_t: caller-owned state of one layer's caches (see hisparse_resolve_noalloc)."""
+    _fields_ = [
+        ("num_requests", ctypes.c_int32), ("cache_slots", ctypes.c_int32), ("top_k", ctypes.c_int32),
+        ("entry_bytes", ctypes.c_int64), ("device", ctypes.c_int32), ("pool_dev", ctypes.c_void_p),
+        ("slot_pos_dev", ctypes.c_void_p), ("last_use_dev", ctypes.c_void_p), ("lru_order_dev", ctypes.c_void_p),
+        ("pos2slot_dev", ctypes.c_void_p), ("capacity_dev", ctypes.c_void_p), ("init_len_dev", ctypes.c_void_p),
+        ("p2s_offset_dev", ctypes.c_void_p), ("host_layer_dev", ctypes.c_void_p), ("resolves_dev", ctypes.c_void_p),
+        ("num_appends_dev", ctypes.c_void_p),
     ]
 
 
@@ -80,6 +93,7 @@ def lib() -> ctypes.CDLL:
             "hisparse_host_free": ([vp], i32),
             "hisparse_host_link_probe": ([i32, sz, i32, P(ctypes.c_double)], i32),
             "hisparse_scatter_read_probe": ([i32, vp, sz, i64, ctypes.c_int32, ctypes.c_int32, i32, P(ctypes.c_double)], i32),
+            "hisparse_resolve_noalloc": ([P(ExternalState), vp, vp, vp, vp, vp, vp], i32),
             "hisparse_strerror": ([i32], ctypes.c_char_p),
             "hisparse_last_cuda_error": ([], i32),
         }
@@ -157,6 +171,21 @@ def scatter_read_probe(host_ptr: int, host_bytes: int, entry_bytes: int, num_rec
     _check(lib().hisparse_scatter_read_probe(device, host_ptr, host_bytes, entry_bytes, num_records, num_ctas, reps,
                                              ctypes.byref(out)), "hisparse_scatter_read_probe")
     return out.value
+
+
+def resolve_noalloc(state: ExternalState, sel, slot_table, hits, misses, status=None, stream=None) -> None:
+    """Resolve on caller-owned state without any device allocation (hisparse_resolve_noalloc).
+
+    For callers that may not call cudaMalloc (all of HBM handed to their own allocator, or a stream capture in
+    progress): every tensor is the caller's; the kernel's scratch is a fixed array inside the library.  Calls
+    on one device share that array, so do not let two of them overlap on the GPU.
+    """
+    n, k = state.num_requests, state.top_k
+    _check(lib().hisparse_resolve_noalloc(ctypes.byref(state), _dev_ptr(sel, "int32", n * k),
+                                          _dev_ptr(slot_table, "int32", n * k), _dev_ptr(hits, "int32", n),
+                                          _dev_ptr(misses, "int32", n),
+                                          status.data_ptr() if status is not None else None, _stream_ptr(stream)),
+           "hisparse_resolve_noalloc")
 
 
 class HiSparse:
