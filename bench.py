@@ -260,7 +260,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     import paper_2608_07009_b200 as hs
-    from paper_2608_07009_b200 import inputs
+    from paper_2608_07009_b200 import inputs, sharding
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -425,15 +425,7 @@ def run_ours(args):
         cyc = st[:, [15, 8, 9, 10, 11, 12, 13, 14]]
         phases["cycles_start_issue_landed_hashed_probed_sync_scanned_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
 
-    if world > 1:
-        t = torch.tensor([total_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_s_max = float(t.item())
-        c = torch.tensor([sel_count], dtype=torch.float64, device=dev)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        sel_total = float(c.item())
-    else:
-        total_s_max, sel_total = total_s, float(sel_count)
+    total_s_max, sel_total = sharding.aggregate(total_s, sel_count, dev)
 
     # ---- e2e: the following steps through the public API with the inputs in pinned host memory ----
     sel_pin = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in sels[n_dev:]]
@@ -462,12 +454,7 @@ def run_ours(args):
                 d2h += cnt_host.numel() * 4
     h2d //= max(1, K)
     d2h //= max(1, K)
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        c = torch.tensor([e2e_sel], dtype=torch.float64, device=dev)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        e2e_s, e2e_sel = float(t.item()), float(c.item())
+    e2e_s, e2e_sel = sharding.aggregate(e2e_s, e2e_sel, dev)
     status |= gpu.status()
     del graphs
     gpu.close()
