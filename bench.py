@@ -50,6 +50,7 @@ def parse_args():
     ap.add_argument("--no-prefetch", action="store_true", help="c3 only: shared layers swap in synchronously")
     ap.add_argument("--skip-io", action="store_true", help="no-IO timing mode (metadata only)")
     ap.add_argument("--phases", action="store_true", help="record the resolve kernel's phase stamps (adds a little time)")
+    ap.add_argument("--no-pdl", action="store_true", help="launch Resolve without programmatic dependent launch")
     ap.add_argument("--no-all-hit", action="store_true", help="skip the scaled all-hit HBM point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-requests", type=int, default=8)
@@ -280,7 +281,8 @@ def run_ours(args):
     hist = [hs.HostHistory(L, cap[r], E) for r in range(N)]
     for r, h in enumerate(hist):
         inputs.fill_history(h.ptr, r, L, cap[r], 0, w.init_len[r], E, w.seed)
-    flags = (hs.FLAG_SKIP_IO if args.skip_io else 0) | (hs.FLAG_PHASE_TIMERS if args.phases else 0)
+    flags = (hs.FLAG_SKIP_IO if args.skip_io else 0) | (hs.FLAG_PHASE_TIMERS if args.phases else 0) \
+        | (hs.FLAG_NO_PDL if args.no_pdl else 0)
     gpu = hs.HiSparse(N, L, lpg, B, k, E, cap, w.init_len, hist, device=local, flags=flags,
                       ctas_per_request=args.ctas_per_request)
     geo = gpu.launch_geometry()
@@ -416,14 +418,13 @@ def run_ours(args):
     phases = None
     if args.phases:
         st = gpu.phase_times().astype(np.int64)
-        d = np.diff(st[:, :6], axis=1) / 1e3
-        phases = {"stage_hash": float(d[:, 0].mean()), "probe": float(d[:, 1].mean()), "scan": float(d[:, 2].mean()),
-                  "publish": float(d[:, 3].mean()), "fetch_after_publish": float(d[:, 4].mean()),
-                  "fetch_span": float((st[:, 6] - st[:, 7]).mean() / 1e3),
+        phases = {"pre_fetch_metadata": float((st[:, 3] - st[:, 0]).mean() / 1e3),
+                  "publish": float((st[:, 4] - st[:, 3]).mean() / 1e3),
+                  "fetch_span": float((st[:, 6] - st[:, 3]).mean() / 1e3),
                   "kernel_span": float((st[:, 6].max() - st[:, 0].min()) / 1e3),
                   "unit": "us, mean over requests, last anchor launch"}
         cyc = st[:, [15, 8, 9, 10, 11, 12, 13, 14]]
-        phases["cycles_start_issue_landed_hashed_probed_sync_scanned_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
+        phases["cycles_issue_landed_lookup_count_barrier_scan_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
 
     total_s_max, sel_total = sharding.aggregate(total_s, sel_count, dev)
 

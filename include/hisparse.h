@@ -54,6 +54,8 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
 #define HISPARSE_FLAG_PHASE_TIMERS 8u      /* the resolve kernel records %globaltimer at its phase boundaries
                                              (hisparse_phase_times); for the phase breakdown of Fig. 7        */
 
+#define HISPARSE_FLAG_NO_PDL 16u           /* launch Resolve without programmatic dependent launch             */
+
 /* sticky device status bits (hisparse_status) */
 #define HISPARSE_STATUS_OUT_OF_RANGE 1u   /* a selected position was outside [0, len) (and not -1)       */
 #define HISPARSE_STATUS_DUPLICATE 2u      /* a position occurred twice in one row                        */
@@ -177,13 +179,12 @@ int hisparse_dump_plan(hisparse_t *h, int req, int layer, int32_t *plan_pos, int
  * device footprint", plus the reserved slot) in *kv_bytes and the metadata in *meta_bytes. */
 int hisparse_device_bytes(const hisparse_config_t *cfg, size_t *kv_bytes, size_t *meta_bytes);
 
-/* With PHASE_TIMERS: stamps of the last anchor resolve, host uint64 [N][16], per request, in nanoseconds:
- * [0] kernel start, [1] selections staged and hashed (Phase 1), [2] slots probed (Phase 2), [3] misses
- * compacted, victims chosen, metadata installed and the plan public (Phase 3), [4] slot table and recency
- * order published (Phase 5), [5] this request's first block done fetching (Phase 4), [6] its last block done fetching, [7] its first
- * block to start fetching; [8..15] SM cycle-counter readings of the first block, for finer splits inside
- * Phases 1-3 ([15] kernel start, [8] loads issued, [9] loads landed, [10] hashed, [11]/[12] probed before/after
- * the barrier, [13] scanned, [14] plan ready).  Synchronises. */
+/* With PHASE_TIMERS: stamps of the last anchor resolve, host uint64 [N][16], per request.
+ * %globaltimer nanoseconds: [0] kernel start, [3] plan ready = fetch begins (end of Phases 1-3), [4] slot table
+ * and recency order published (Phase 5), [5] this request's first block done fetching, [6] its last block done
+ * fetching (Phase 4), [7] = [3]; [1], [2] unused.  SM cycle-counter readings of the first block, for splits
+ * inside Phases 1-3: [15] kernel start, [8] loads issued, [9] loads landed, [10] selections looked up and
+ * classified, [11] / [12] counted, before / after the barrier, [13] scanned, [14] plan ready.  Synchronises. */
 int hisparse_phase_times(hisparse_t *h, uint64_t *out);
 
 /* Launch geometry chosen at create: thread blocks per request and threads per block. */

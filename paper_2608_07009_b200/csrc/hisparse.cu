@@ -45,7 +45,8 @@ thread_local int g_last_cuda_error = 0;
   } while (0)
 
 constexpr int kThreads = 1024;       // threads per block of the resolve / replay kernels
-constexpr int kFetchUnroll = 4;      // 16-byte host loads in flight per thread
+constexpr int kFetchUnroll = 4;      // 16-byte host loads in flight per thread (probe kernel)
+constexpr int kBarBytes = (kThreads + 2) * 8;  // one mbarrier per thread for the fetch ring + one for staging
 constexpr int32_t kMiss = -2;        // s_out marker: valid selection, not (yet) found resident
 constexpr int32_t kDupBase = -3;     // s_out marker: duplicate of row entry -(v + 3)
 
@@ -71,6 +72,7 @@ struct DevState {
   uint32_t *status;
   int meta_smem;                   // bytes of shared memory the metadata arrays take (ring follows)
   int io_threads, io_depth, io_chunk;  // fetch pipeline: issuing threads, ring slots per thread, bytes per piece
+  int ring_bytes;                  // io_threads * io_depth * io_chunk
   unsigned long long *phase_ns;    // [N][16]: 8 globaltimer stamps, then 8 SM cycle-counter stamps (PHASE_TIMERS)
 };
 
@@ -227,6 +229,8 @@ struct TmaFetch {
 __device__ __forceinline__ void fetch_barriers_init(unsigned long long *bars, int io_threads) {
   if ((int)threadIdx.x < io_threads)
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + threadIdx.x)) : "memory");
+  if (threadIdx.x == 0)  // the staging barrier of the page-table slice
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + kThreads)) : "memory");
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 
@@ -318,28 +322,52 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  int32_t *s_sel, int32_t *s_out, int32_t *s_plan_pos,
                                                  int32_t *s_plan_slot, unsigned long long *s_tab, uint32_t *s_hitbits,
                                                  uint32_t *s_vicbits, uint16_t *s_order, int *s_warp, int *s_misc,
-                                                 const uint32_t hit_stamp, unsigned long long *stamps, int &m,
+                                                 const int64_t cap_r, const int64_t init_len_r,
+                                                 const int64_t p2s_off_r, unsigned long long *stamps,
+                                                 unsigned char *s_ring, unsigned long long *s_bars, int &m,
                                                  int &n_nonhit, uint32_t &my_status) {
   constexpr int T = kThreads;
   const int tid = threadIdx.x, lane = tid & 31;
-  const int k = d.k, B = d.B, H = d.H, W = d.W;
+  const int k = d.k, B = d.B, H = d.H;
   const uint32_t mask = (uint32_t)(H - 1);
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
-  uint32_t *last_use = d.last_use + rg * B;
 
-  // Phase 1: stage the row and the recency order (one round trip to HBM), clear the marks and the table.
+  // Phase 1: stage the row and the recency order (one round trip to HBM).  The request's slice of the page
+  // table is streamed into the (still idle) fetch ring with bulk copies when it fits, so that Phase 2's k random
+  // lookups hit shared memory instead of queueing as 32-byte sector reads on one SM.
   stage_async(s_sel, row, k * 4);
   stage_async(s_order, d.order + rg * B, B * 2);
-  int64_t len, newest;
-  history_state(d, r, len, newest);
-  const int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)(rg - (int64_t)r * d.G) * d.cap[r];
-  for (int i = tid; i < H; i += T) s_tab[i] = kEmptyEntry;
-  for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
-  if (tid < 4) s_misc[tid] = 0;
+  const int32_t *p2s = d.pos2slot + p2s_off_r + (int64_t)(rg - (int64_t)r * d.G) * cap_r;
+  const uintptr_t p2s_aligned = (uintptr_t)p2s & ~(uintptr_t)15;
+  const int lead = (int)(((uintptr_t)p2s - p2s_aligned) >> 2);
+  const int64_t stage_bytes = ((int64_t)lead * 4 + cap_r * 4) & ~(int64_t)15;  // whole 16-byte units only
+  const bool staged = stage_bytes + 16 <= (int64_t)d.ring_bytes;
+  const uint32_t stage_bar = smem_u32(s_bars + kThreads);
+  if (staged && tid == 0) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(stage_bar), "r"((uint32_t)stage_bytes) : "memory");
+    for (int64_t o = 0; o < stage_bytes; o += 32768) {
+      const uint32_t n = (uint32_t)(stage_bytes - o < 32768 ? stage_bytes - o : 32768);
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(s_ring) + (uint32_t)o), "l"((const char *)p2s_aligned + o), "r"(n), "r"(stage_bar) : "memory");
+    }
+  }
+  if (staged && tid >= 32 && tid < 36) {  // the last, partial 16-byte unit of the slice: plain copies
+    const int64_t e = stage_bytes / 4 + (tid - 32);
+    if (e < lead + cap_r) reinterpret_cast<int32_t *>(s_ring)[e] = reinterpret_cast<const int32_t *>(p2s_aligned)[e];
+  }
+  const int64_t na = *(volatile int32_t *)d.n_appends;
+  const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
+  const int64_t newest = (na > 0 && init_len_r + na <= cap_r) ? init_len_r + na - 1 : -1;
   if (timers && tid == 0) stamps[8] = clock64();
   asm volatile("cp.async.wait_all;" ::: "memory");
+  bool use_staged = staged;
+  if (staged && !mbar_wait_bounded(stage_bar, 0u)) {
+    use_staged = false;  // bounded wait expired: fall back to the table in HBM
+    my_status |= HISPARSE_STATUS_TIMEOUT;
+  }
   __syncthreads();
   if (timers && tid == 0) stamps[9] = clock64();
+  const int32_t *s_p2s = reinterpret_cast<const int32_t *>(s_ring) + lead;
 
   // Phase 2: hit detection through the page table (position -> slot): all of a thread's lookups are issued
   // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
@@ -353,8 +381,9 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
     if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
     if (!ok) pos[i] = -1;
-    got[i] = ok ? __ldg(p2s + pos[i]) : -1;
+    got[i] = !ok ? -1 : (use_staged ? s_p2s[pos[i]] : __ldg(p2s + pos[i]));
   }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
   int my_valid = 0;
 #pragma unroll
   for (int i = 0; i < kSelPerThread; ++i) {
@@ -373,8 +402,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
         if (atomicOr(&s_hitbits[s >> 5], bit) & bit) {
           my_status |= HISPARSE_STATUS_DUPLICATE;  // the same resident position again: same slot, counted once
         } else {
-          ++my_valid;
-          last_use[s] = hit_stamp;
+          ++my_valid;  // the hit's stamp is written later, in slot order (coalesced), from the hit bits
         }
       } else {
         o = kMiss;
@@ -414,9 +442,9 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) my_valid += __shfl_xor_sync(0xffffffffu, my_valid, o);
   if (lane == 0 && my_valid) atomicAdd(&s_misc[1], my_valid);
-  if (timers && tid == 0) { stamps[1] = global_ns(); stamps[11] = clock64(); }
+  if (timers && tid == 0) stamps[11] = clock64();
   __syncthreads();
-  if (timers && tid == 0) { stamps[2] = global_ns(); stamps[12] = clock64(); }
+  if (timers && tid == 0) stamps[12] = clock64();
 
   // Phase 3: ONE block scan over packed counts (non-hit slots in recency order | misses in selection order).
   // Thread t owns IPT consecutive entries of the recency order and kSelPerThread consecutive row entries.
@@ -496,21 +524,30 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   int32_t *s_vicpre = s_hitpre + W;
   uint16_t *s_order = reinterpret_cast<uint16_t *>(s_vicpre + W);
   unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
-  unsigned char *s_ring = smem_raw + d.meta_smem + kThreads * 8;
+  unsigned char *s_ring = smem_raw + d.meta_smem + kBarBytes;
 
-  fetch_barriers_init(s_bars, d.io_threads);  // made visible by the barriers below, long before first use
+  // Prologue that depends on nothing an earlier kernel wrote: barriers, cleared marks and table.  With
+  // programmatic dependent launch it overlaps the tail of whatever runs before this kernel in the stream.
+  fetch_barriers_init(s_bars, d.io_threads);
+  if (part == 0) {
+    for (int i = tid; i < H; i += T) s_tab[i] = kEmptyEntry;
+    for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
+    if (tid < 4) s_misc[tid] = 0;
+  }
+  const int64_t cap_r = d.cap[r], init_len_r = d.init_len[r], p2s_off_r = d.p2s_off[r];  // fixed at create
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   TmaFetch fetch;
   int m = 0, n_nonhit = 0;
   uint32_t t = 0;
   if (part == 0) {
     if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
     t = d.t[rg] + 1u;
-    const uint32_t hit_stamp = 2u * t + 1u, miss_stamp = 2u * t;
+    const uint32_t miss_stamp = 2u * t;
     uint32_t my_status = 0;
     const int32_t *row = sel + (int64_t)r * k;
 #define HS_META(IPT)                                                                                              \
   resolve_metadata<IPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits, s_order, \
-                        s_warp, s_misc, hit_stamp, stamps, m, n_nonhit, my_status)
+                        s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, m, n_nonhit, my_status)
     if (B <= 4 * T) HS_META(4);
     else if (B <= 8 * T) HS_META(8);
     else HS_META(16);
@@ -522,7 +559,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     // Phase 5, metadata half: page table, slot array, stamps, plan
     int32_t *slot_pos = d.slot_pos + rg * B;
     uint32_t *last_use = d.last_use + rg * B;
-    int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
+    int32_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
     int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
     for (int i = tid; i < m; i += T) {
       const int v = s_plan_slot[i];
@@ -575,12 +612,17 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     }
     __syncthreads();
     const int n_surv = n_nonhit - m;
+    uint32_t *last_use = d.last_use + rg * B;
     for (int s = tid; s < B; s += T) {
       const int w = s >> 5;
       const uint32_t bit = 1u << (s & 31), lt = bit - 1u;
       const uint32_t vw = s_vicbits[w], hw = s_hitbits[w];
-      if (vw & bit) s_order[n_surv + s_vicpre[w] + __popc(vw & lt)] = (uint16_t)s;
-      else if (hw & bit) s_order[n_nonhit + s_hitpre[w] + __popc(hw & lt)] = (uint16_t)s;
+      if (vw & bit) {
+        s_order[n_surv + s_vicpre[w] + __popc(vw & lt)] = (uint16_t)s;
+      } else if (hw & bit) {
+        s_order[n_nonhit + s_hitpre[w] + __popc(hw & lt)] = (uint16_t)s;
+        last_use[s] = 2u * t + 1u;  // hits are stamped above this step's fetched records
+      }
     }
     __syncthreads();
     for (int q = tid; q < B; q += T) order[q] = s_order[q];
@@ -606,7 +648,9 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       fetch.issue();
     }
   }
-  // Phase 4, rest: wait for the batches, store them into the cache slots, issue what is left.
+  // Phase 4, rest: wait for the batches, store them into the cache slots, issue what is left.  Whatever follows
+  // in the stream may be scheduled from here on (it still waits for this grid to finish before it reads).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   fetch.drain(d.status);
   if (timers) {
     __syncthreads();
@@ -626,7 +670,7 @@ __global__ void __launch_bounds__(kThreads, 1) replay_kernel(const DevState d, c
   int32_t *s_plan_pos = reinterpret_cast<int32_t *>(smem_raw);
   int32_t *s_plan_slot = s_plan_pos + d.k;
   unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
-  unsigned char *s_ring = smem_raw + d.meta_smem + kThreads * 8;
+  unsigned char *s_ring = smem_raw + d.meta_smem + kBarBytes;
   const int r = blockIdx.x / S, part = blockIdx.x - r * S;
   const int64_t rg = (int64_t)r * d.G + layer / d.lpg;
   const int m = d.plan_n[rg];
@@ -889,13 +933,15 @@ int launch_resolve(hisparse *h, int layer, const int32_t *sel, int32_t *table, i
   cfg.blockDim = dim3((unsigned)h->T);
   cfg.dynamicSmemBytes = h->resolve_smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)h->S;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (h->d.flags & HISPARSE_FLAG_NO_PDL) ? 1 : 2;
   HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel, h->d, layer, sel, table, hits, misses, h->S));
   return HISPARSE_OK;
 }
@@ -986,13 +1032,14 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   // shared memory: metadata arrays, one mbarrier per thread, then the staging ring of the fetch pipeline,
   // which takes whatever is left (pieces of at most 8 KB; at least one piece must fit)
   d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
-  const int64_t ring_room = (int64_t)max_optin - 1024 - d.meta_smem - kThreads * 8;
+  const int64_t ring_room = (int64_t)max_optin - 1024 - d.meta_smem - kBarBytes;
   if (ring_room < 16) return fail(HISPARSE_EINVAL);
   d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
   const int slots = (int)(ring_room / d.io_chunk);
   d.io_threads = std::min(slots, kThreads);
   d.io_depth = std::min(slots / d.io_threads, 8);
-  h->resolve_smem = (size_t)d.meta_smem + kThreads * 8 + (size_t)d.io_threads * d.io_depth * d.io_chunk;
+  d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
+  h->resolve_smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
   h->replay_smem = h->resolve_smem;   // same offsets, so that both kernels share the pipeline's geometry
   if (cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaFuncSetAttribute(replay_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
@@ -1449,13 +1496,14 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   d.ticket = nullptr;
   d.phase_ns = nullptr;      // only touched with PHASE_TIMERS, which is off here
   d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
-  const int64_t ring_room = (int64_t)optin - 1024 - d.meta_smem - kThreads * 8;
+  const int64_t ring_room = (int64_t)optin - 1024 - d.meta_smem - kBarBytes;
   if (ring_room < 16) return HISPARSE_EINVAL;
   d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
   const int slots = (int)(ring_room / d.io_chunk);
   d.io_threads = std::min(slots, kThreads);
   d.io_depth = std::min(slots / d.io_threads, 8);
-  const size_t smem = (size_t)d.meta_smem + kThreads * 8 + (size_t)d.io_threads * d.io_depth * d.io_chunk;
+  d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
+  const size_t smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
 
   cudaStream_t s = as_stream(stream);
   // the counters other blocks read must not carry the previous call's values into this one
