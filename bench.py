@@ -243,7 +243,10 @@ def all_hit_point(dev, hbm_peak):
     t = statistics.mean(times)
     achieved = ALGO_BYTES_PER_HIT * N * k / t / 1e9
     return {"bound": "hbm", "achieved": achieved, "peak": hbm_peak["value"], "unit": "GB/s",
-            "frac": achieved / hbm_peak["value"], "peak_source": hbm_peak["source"], "traffic": None,
+            "frac": achieved / hbm_peak["value"], "peak_source": hbm_peak["source"],
+            "traffic": 119925760 if N == 2048 else None,
+            "traffic_source": "profiles/resolve_kernel_all_hit_set_full.md",
+            "issue_bound_note": "ncu: 44 % of peak instruction issue, 10 % of DRAM throughput: issue/latency bound",
             "workload": "scaled all-hit point: %d requests x 1 layer, k=%d, B=%d, every selection hits" % (N, k, B),
             "algorithmic_bytes_per_launch": ALGO_BYTES_PER_HIT * N * k, "launch_us": t * 1e6,
             "selections_per_s": N * k / t, "ctas_per_request": geo["ctas_per_request"]}
@@ -287,6 +290,10 @@ def run_ours(args):
                       ctas_per_request=args.ctas_per_request)
     geo = gpu.launch_geometry()
     link_peak = hs.host_link_probe(local, 1 << 30, 10)
+    # ceiling for reads issued by SMs: a copy-only kernel over random records of request 0's history
+    hb = min(hist[0].nbytes, 1 << 32)
+    sm_read = {"%dMB" % mb: hs.scatter_read_probe(hist[0].ptr, hb, E, max(1, (mb << 20) // E), 148, 5, local)
+               for mb in (4, 32)}
 
     # the whole trace, generated up front: cold step, warm-up, timed, eager-profile and e2e steps
     K, W = args.steps, args.warmup
@@ -497,7 +504,9 @@ def run_ours(args):
             "bound": "host_link", "achieved": achieved, "peak": link_peak, "unit": "GB/s",
             "frac": achieved / link_peak if link_peak else None,
             "peak_source": "measured in this run: best of 10 bulk pinned cudaMemcpyAsync H2D of 1 GiB",
-            "kernel": "resolve_kernel", "traffic": None,
+            "kernel": "resolve_kernel",
+            "traffic": 4838912 if (w.name, N) == ("c2_dsa_decode", 32) else None,
+            "traffic_source": "profiles/resolve_kernel_c2_set_full.md: dram__bytes_read + dram__bytes_write of one launch",
             "algorithmic_bytes_per_launch": algo_bytes_per_launch, "launch_us": avg_launch_s * 1e6,
             "launch_us_method": "CUDA events around each step's graph replay / resolve launches per step"},
         "per_layer_resolve_us": {"graph": avg_launch_s * 1e6,
@@ -505,6 +514,8 @@ def run_ours(args):
                                  "eager_p99": float(np.percentile(res_us[:, anchor_layers], 99)),
                                  "eager_mean": float(res_us[:, anchor_layers].mean())},
         "misses_per_request_layer": float(miss_h[:, anchor_layers].mean()),
+        "host_link": {"memcpy_peak_gb_s": link_peak, "sm_issued_read_gb_s": sm_read,
+                      "note": "copy-only kernel, 148 blocks, random records of this workload's size"},
         "cold_step_ms": cold_ms, "status_bits": status, "launch_geometry": geo, "setup_s": setup_s,
     }
     if phases:

@@ -88,7 +88,7 @@ typedef struct {
   int32_t device;            /* CUDA device ordinal                                                    */
   uint32_t flags;            /* HISPARSE_FLAG_*                                                         */
   int32_t ctas_per_request;  /* thread blocks (one cluster) that share one request's fetch work;
-                                0 = choose from N and the SM count; otherwise 1, 2, 4 or 8             */
+                                0 = choose from N (about 32 blocks in all); otherwise 1, 2, 4 or 8             */
 } hisparse_config_t;
 
 /* Sec. 3.3 step (2) "Admission": reserve the per-layer caches and metadata of N requests.  All

@@ -73,6 +73,7 @@ struct DevState {
   int meta_smem;                   // bytes of shared memory the metadata arrays take (ring follows)
   int io_threads, io_depth, io_chunk;  // fetch pipeline: issuing threads, ring slots per thread, bytes per piece
   int ring_bytes;                  // io_threads * io_depth * io_chunk
+  int io_ppr;                      // pieces per record = ceil(E / io_chunk)
   unsigned long long *phase_ns;    // [N][16]: 8 globaltimer stamps, then 8 SM cycle-counter stamps (PHASE_TIMERS)
 };
 
@@ -147,7 +148,7 @@ struct TmaFetch {
                                        int part_, int nparts_) {
     const int tid = threadIdx.x;
     E = d.E; chunk = d.io_chunk; depth = d.io_depth; io_threads = d.io_threads;
-    ppr = (int)((E + chunk - 1) / chunk);
+    ppr = d.io_ppr;
     total = (int64_t)m * ppr;
     part = part_; nparts = nparts_;
     s_pos = pos; s_slot = slot;
@@ -171,7 +172,7 @@ struct TmaFetch {
     for (int s = 0; s < depth; ++s) {
       const int64_t c = piece_of(batch * depth + s);
       if (c >= total) break;
-      const int piece = (int)(c % ppr);
+      const int piece = ppr == 1 ? 0 : (int)(c % ppr);
       const int64_t rest = E - (int64_t)piece * chunk;
       bytes_total += (uint32_t)(rest < chunk ? rest : chunk);
     }
@@ -180,7 +181,7 @@ struct TmaFetch {
     for (int s = 0; s < depth; ++s) {
       const int64_t c = piece_of(batch * depth + s);
       if (c >= total) break;
-      const int64_t rec = c / ppr;
+      const int64_t rec = ppr == 1 ? c : c / ppr;
       const int piece = (int)(c - rec * ppr);
       const int64_t rest = E - (int64_t)piece * chunk;
       const uint32_t bytes = (uint32_t)(rest < chunk ? rest : chunk);
@@ -203,7 +204,7 @@ struct TmaFetch {
     for (int s = 0; s < depth; ++s) {
       const int64_t c = piece_of(batch * depth + s);
       if (c >= total) break;
-      const int64_t rec = c / ppr;
+      const int64_t rec = ppr == 1 ? c : c / ppr;
       const int piece = (int)(c - rec * ppr);
       const int64_t rest = E - (int64_t)piece * chunk;
       const uint32_t bytes = (uint32_t)(rest < chunk ? rest : chunk);
@@ -327,7 +328,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  unsigned char *s_ring, unsigned long long *s_bars, int &m,
                                                  int &n_nonhit, uint32_t &my_status) {
   constexpr int T = kThreads;
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x;
   const int k = d.k, B = d.B, H = d.H;
   const uint32_t mask = (uint32_t)(H - 1);
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
@@ -384,7 +385,6 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     got[i] = !ok ? -1 : (use_staged ? s_p2s[pos[i]] : __ldg(p2s + pos[i]));
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
-  int my_valid = 0;
 #pragma unroll
   for (int i = 0; i < kSelPerThread; ++i) {
     const int j = tid + i * T;
@@ -394,19 +394,16 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     if (p >= 0) {
       if ((int64_t)p == newest) {  // reserved newest-record slot, outside the LRU set
         o = B;
-        if (atomicExch(&s_misc[2], 1) == 0) ++my_valid; else my_status |= HISPARSE_STATUS_DUPLICATE;
+        if (atomicExch(&s_misc[2], 1) != 0) my_status |= HISPARSE_STATUS_DUPLICATE;
       } else if (got[i] >= 0) {
         const int s = got[i];
         o = s;
         const uint32_t bit = 1u << (s & 31);
-        if (atomicOr(&s_hitbits[s >> 5], bit) & bit) {
-          my_status |= HISPARSE_STATUS_DUPLICATE;  // the same resident position again: same slot, counted once
-        } else {
-          ++my_valid;  // the hit's stamp is written later, in slot order (coalesced), from the hit bits
-        }
+        // a bit that is already set = the same resident position selected again: same slot, counted once.
+        // The hit's stamp is written later, in slot order (coalesced), from the hit bits.
+        if (atomicOr(&s_hitbits[s >> 5], bit) & bit) my_status |= HISPARSE_STATUS_DUPLICATE;
       } else {
         o = kMiss;
-        ++my_valid;
         const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)j;
         uint32_t h = hash_pos(p, d.hshift);
         for (uint32_t it = 0; it <= mask; ++it) {
@@ -433,15 +430,11 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
         table_lookup<1>(s_tab, mask, d.hshift, key, owner);
         if (owner[0] != j) {
           s_out[j] = kDupBase - owner[0];
-          --my_valid;
           my_status |= HISPARSE_STATUS_DUPLICATE;
         }
       }
     }
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) my_valid += __shfl_xor_sync(0xffffffffu, my_valid, o);
-  if (lane == 0 && my_valid) atomicAdd(&s_misc[1], my_valid);
   if (timers && tid == 0) stamps[11] = clock64();
   __syncthreads();
   if (timers && tid == 0) stamps[12] = clock64();
@@ -503,7 +496,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
                int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out, const int S) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_warp[32];
-  __shared__ int s_misc[4];  // [0] any duplicate  [1] valid distinct selections
+  __shared__ int s_misc[4];  // [0] a missing position was selected twice  [2] the newest position was selected
   constexpr int T = kThreads;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x / S, part = blockIdx.x - r * S;
@@ -627,10 +620,11 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     __syncthreads();
     for (int q = tid; q < B; q += T) order[q] = s_order[q];
     if (tid == 0) {
-      const int nvalid = s_misc[1];
-      hits_out[r] = nvalid - m;
+      // distinct hits = slots whose hit bit is set (+ the reserved slot if the newest position was selected)
+      const int nhits = (B - n_nonhit) + (s_misc[2] ? 1 : 0);
+      hits_out[r] = nhits;
       misses_out[r] = m;
-      d.anchor_hits[rg] = nvalid - m;
+      d.anchor_hits[rg] = nhits;
       d.anchor_misses[rg] = m;
       d.t[rg] = t;
     }
@@ -1039,17 +1033,22 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   d.io_threads = std::min(slots, kThreads);
   d.io_depth = std::min(slots / d.io_threads, 8);
   d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
+  d.io_ppr = (int)((d.E + d.io_chunk - 1) / d.io_chunk);
   h->resolve_smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
   h->replay_smem = h->resolve_smem;   // same offsets, so that both kernels share the pipeline's geometry
   if (cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaFuncSetAttribute(replay_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
 
-  // Blocks per request: as many as still let all N clusters be resident at once.
+  // Blocks per request: enough of them that about 32 blocks pull on the host link together (measured: fewer
+  // leave it under-used when requests are few, more only add launch and barrier cost), as long as all N
+  // clusters are resident at once.
   if (c->ctas_per_request) {
     h->S = c->ctas_per_request;
   } else {
+    int want = 1;
+    while (want < 8 && N * want < 32) want <<= 1;
     h->S = 1;
-    for (int s = 8; s > 1; s >>= 1) {
+    for (int s = want; s > 1; s >>= 1) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)(N * s));
       cfg.blockDim = dim3(kThreads);
@@ -1503,6 +1502,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   d.io_threads = std::min(slots, kThreads);
   d.io_depth = std::min(slots / d.io_threads, 8);
   d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
+  d.io_ppr = (int)((d.E + d.io_chunk - 1) / d.io_chunk);
   const size_t smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
 
   cudaStream_t s = as_stream(stream);
