@@ -248,7 +248,7 @@ typedef struct {
   int32_t *slot_pos_dev;         /* int32 [N][B]                                                          */
   uint32_t *last_use_dev;        /* uint32 [N][B]                                                         */
   uint16_t *lru_order_dev;       /* uint16 [N][B]                                                         */
-  int32_t *pos2slot_dev;         /* int32, request r's page table at [p2s_offset[r], p2s_offset[r] + capacity[r]) */
+  int16_t *pos2slot_dev;         /* int16, request r's page table at [p2s_offset[r], p2s_offset[r] + capacity[r]) */
   const int64_t *capacity_dev;   /* int64 [N]                                                             */
   const int64_t *init_len_dev;   /* int64 [N]: history length before any append                           */
   const int64_t *p2s_offset_dev; /* int64 [N]                                                             */

@@ -7,7 +7,7 @@
 //   last_use  uint32 [N][G][B]        recency stamps: 2t+1 hit at resolve t, 2t fetched at resolve t, 0 unused
 //   order     uint16 [N][G][B]        slots from least to most recent; always equal to sorting the slots by
 //                                     (last_use, slot).  Kept so that victim choice is a prefix scan, not a sort
-//   pos2slot  int32  ragged [N][G][capacity[r]]  the page table (Sec. 3.2), -1 = host-only
+//   pos2slot  int16  ragged [N][G][capacity[r]]  the page table (Sec. 3.2), -1 = host-only
 //   plan_*    int32  [N][G][k]        miss plan of the last anchor resolve (Sec. 3.5)
 // All step-dependent scalars (resolve counters, number of appends, plan sizes) live in device memory so
 // that every launch is replayable from a CUDA graph.
@@ -61,7 +61,7 @@ struct DevState {
   int32_t *slot_pos;
   uint32_t *last_use;
   uint16_t *order;
-  int32_t *pos2slot;
+  int16_t *pos2slot;               // page table entries are slots (< 16384) or -1
   const int64_t *cap, *init_len, *p2s_off;
   uint8_t *const *host;
   uint32_t *t;
@@ -223,7 +223,8 @@ struct TmaFetch {
       complete(status);
       pending = issue();
     }
-    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    // complete() already waited until every store of this thread had read its ring slot (wait_group.read), which
+    // is what shared memory needs before the block exits; the writes themselves are complete at grid end.
   }
 };
 
@@ -338,10 +339,10 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   // lookups hit shared memory instead of queueing as 32-byte sector reads on one SM.
   stage_async(s_sel, row, k * 4);
   stage_async(s_order, d.order + rg * B, B * 2);
-  const int32_t *p2s = d.pos2slot + p2s_off_r + (int64_t)(rg - (int64_t)r * d.G) * cap_r;
+  const int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)(rg - (int64_t)r * d.G) * cap_r;
   const uintptr_t p2s_aligned = (uintptr_t)p2s & ~(uintptr_t)15;
-  const int lead = (int)(((uintptr_t)p2s - p2s_aligned) >> 2);
-  const int64_t stage_bytes = ((int64_t)lead * 4 + cap_r * 4) & ~(int64_t)15;  // whole 16-byte units only
+  const int lead = (int)(((uintptr_t)p2s - p2s_aligned) >> 1);
+  const int64_t stage_bytes = ((int64_t)lead * 2 + cap_r * 2) & ~(int64_t)15;  // whole 16-byte units only
   const bool staged = stage_bytes + 16 <= (int64_t)d.ring_bytes;
   const uint32_t stage_bar = smem_u32(s_bars + kThreads);
   if (staged && tid == 0) {
@@ -352,9 +353,9 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                    ::"r"(smem_u32(s_ring) + (uint32_t)o), "l"((const char *)p2s_aligned + o), "r"(n), "r"(stage_bar) : "memory");
     }
   }
-  if (staged && tid >= 32 && tid < 36) {  // the last, partial 16-byte unit of the slice: plain copies
-    const int64_t e = stage_bytes / 4 + (tid - 32);
-    if (e < lead + cap_r) reinterpret_cast<int32_t *>(s_ring)[e] = reinterpret_cast<const int32_t *>(p2s_aligned)[e];
+  if (staged && tid >= 32 && tid < 40) {  // the last, partial 16-byte unit of the slice: plain copies
+    const int64_t e = stage_bytes / 2 + (tid - 32);
+    if (e < lead + cap_r) reinterpret_cast<int16_t *>(s_ring)[e] = reinterpret_cast<const int16_t *>(p2s_aligned)[e];
   }
   const int64_t na = *(volatile int32_t *)d.n_appends;
   const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
@@ -368,7 +369,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   }
   __syncthreads();
   if (timers && tid == 0) stamps[9] = clock64();
-  const int32_t *s_p2s = reinterpret_cast<const int32_t *>(s_ring) + lead;
+  const int16_t *s_p2s = reinterpret_cast<const int16_t *>(s_ring) + lead;
 
   // Phase 2: hit detection through the page table (position -> slot): all of a thread's lookups are issued
   // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
@@ -382,7 +383,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
     if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
     if (!ok) pos[i] = -1;
-    got[i] = !ok ? -1 : (use_staged ? s_p2s[pos[i]] : __ldg(p2s + pos[i]));
+    got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : __ldg(p2s + pos[i]));
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
 #pragma unroll
@@ -552,7 +553,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     // Phase 5, metadata half: page table, slot array, stamps, plan
     int32_t *slot_pos = d.slot_pos + rg * B;
     uint32_t *last_use = d.last_use + rg * B;
-    int32_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
+    int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
     int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
     for (int i = tid; i < m; i += T) {
       const int v = s_plan_slot[i];
@@ -560,7 +561,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       const int32_t old = slot_pos[v];
       if (old >= 0) p2s[old] = -1;
       slot_pos[v] = p;
-      p2s[p] = v;
+      p2s[p] = (int16_t)v;
       last_use[v] = miss_stamp;
       plan_pos_g[i] = p;
       plan_slot_g[i] = v;
@@ -793,7 +794,7 @@ __global__ void validate_kernel(const DevState d, const int g) {
   const int32_t *slot_pos = d.slot_pos + rg * B;
   const uint32_t *last_use = d.last_use + rg * B;
   const uint16_t *order = d.order + rg * B;
-  const int32_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
+  const int16_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
   for (int i = threadIdx.x; i < d.W; i += blockDim.x) seen[i] = 0u;
   __syncthreads();
   bool bad = false;
@@ -976,7 +977,7 @@ int hisparse_device_bytes(const hisparse_config_t *c, size_t *kv_bytes, size_t *
     size_t cap_sum = 0;
     for (size_t r = 0; r < N; ++r) cap_sum += (size_t)c->capacity[r];
     *meta_bytes = N * G * B * (4 + 4 + 2)          /* slot_pos, last_use, order */
-                  + cap_sum * G * 4                 /* page tables */
+                  + cap_sum * G * 2                 /* page tables */
                   + N * G * k * 4 * 3               /* plan_pos, plan_slot, anchor_out */
                   + N * G * 4 * 4                   /* t, plan_n, anchor hits / misses */
                   + N * (8 * 3 + 8) + 16;           /* cap, init_len, p2s_off, host pointers, scalars */
@@ -1096,7 +1097,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRYC(cudaMemset(d.pool, 0, (size_t)L * d.layer_pool_bytes));
   HS_TRYC(cudaMemset(d.slot_pos, 0xff, NG * B * 4));
   HS_TRYC(cudaMemset(d.last_use, 0, NG * B * 4));
-  HS_TRYC(cudaMemset(d.pos2slot, 0xff, (size_t)h->p2s_total * 4));
+  HS_TRYC(cudaMemset(d.pos2slot, 0xff, (size_t)h->p2s_total * 2));
   HS_TRYC(cudaMemset(d.t, 0, NG * 4));
   HS_TRYC(cudaMemset(d.plan_n, 0, NG * 4));
   HS_TRYC(cudaMemset(d.anchor_out, 0xff, NG * k * 4));
@@ -1288,9 +1289,12 @@ int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, ui
     HS_CUDA(cudaMemcpy(tmp.data(), h->d.order + rg * B, (size_t)B * 2, cudaMemcpyDeviceToHost));
     for (int i = 0; i < B; ++i) lru_order[i] = tmp[i];
   }
-  if (pos2slot)
-    HS_CUDA(cudaMemcpy(pos2slot, h->d.pos2slot + h->p2s_off[req] + (int64_t)g * h->cap[req], (size_t)h->cap[req] * 4,
+  if (pos2slot) {
+    std::vector<int16_t> tmp((size_t)h->cap[req]);
+    HS_CUDA(cudaMemcpy(tmp.data(), h->d.pos2slot + h->p2s_off[req] + (int64_t)g * h->cap[req], (size_t)h->cap[req] * 2,
                        cudaMemcpyDeviceToHost));
+    for (int64_t i = 0; i < h->cap[req]; ++i) pos2slot[i] = tmp[(size_t)i];
+  }
   int32_t na = 0;
   HS_CUDA(cudaMemcpy(&na, h->d.n_appends, 4, cudaMemcpyDeviceToHost));
   const int64_t il = h->init_len[req], cap = h->cap[req];

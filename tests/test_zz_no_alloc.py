@@ -36,7 +36,7 @@ def test_noalloc_matches_handle_on_two_calls():
     last_use = torch.zeros((N, B), dtype=torch.int32, device=dev)          # uint32 bit patterns
     order = torch.arange(B, dtype=torch.int16, device=dev).repeat(N, 1).contiguous()   # uint16 bit patterns
     offs = np.concatenate([[0], np.cumsum(cap)[:-1]]).astype(np.int64)
-    pos2slot = torch.full((int(sum(cap)),), -1, dtype=torch.int32, device=dev)
+    pos2slot = torch.full((int(sum(cap)),), -1, dtype=torch.int16, device=dev)
     cap_d = torch.tensor(cap, dtype=torch.int64, device=dev)
     len_d = torch.tensor(lens, dtype=torch.int64, device=dev)
     off_d = torch.from_numpy(offs).to(dev)
@@ -74,7 +74,7 @@ def test_noalloc_matches_handle_on_two_calls():
                 assert np.array_equal(slot_pos[r].cpu().numpy(), s["slot_pos"])
                 assert np.array_equal(last_use[r].cpu().numpy().view(np.uint32), s["last_use"])
                 assert np.array_equal(order[r].cpu().numpy().view(np.uint16).astype(np.int32), s["lru_order"])
-                assert np.array_equal(pos2slot[offs[r]:offs[r] + cap[r]].cpu().numpy(), s["pos2slot"])
+                assert np.array_equal(pos2slot[offs[r]:offs[r] + cap[r]].cpu().numpy().astype(np.int32), s["pos2slot"])
                 assert int(resolves[r]) == s["resolves"] == call + 1
         assert int(status.item()) == 0 and ref.status() == 0
         # sizes beyond the fixed scratch are refused with their own error code, before anything is enqueued
