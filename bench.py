@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--overlap", type=float, default=0.9, help="c3 only: step-to-step selection overlap")
     ap.add_argument("--requests", type=int, default=0, help="override the number of requests (reduced runs)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (reduced runs)")
+    ap.add_argument("--cache-slots", type=int, default=0, help="override B (cache-size sweeps)")
+    ap.add_argument("--top-k", type=int, default=0, help="override k")
     ap.add_argument("--ctas-per-request", type=int, default=0)
     ap.add_argument("--no-prefetch", action="store_true", help="c3 only: shared layers swap in synchronously")
     ap.add_argument("--skip-io", action="store_true", help="no-IO timing mode (metadata only)")
@@ -78,6 +80,11 @@ def make_workload(args, rank: int = 0):
         w.num_requests = args.requests
     if args.layers:
         w.num_layers = args.layers
+    if args.cache_slots:
+        w.cache_slots = args.cache_slots
+    if args.top_k:
+        w.keep = round(w.keep * args.top_k / w.top_k)
+        w.top_k = args.top_k
     return w
 
 

@@ -63,6 +63,16 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
 #define HISPARSE_STATUS_INCONSISTENT 8u   /* DEBUG_VALIDATE found broken metadata                        */
 #define HISPARSE_STATUS_TIMEOUT 16u       /* a bounded device-side wait expired                          */
 
+/* replacement policies (hisparse_config_t.policy).  LRU with hits ranked above the step's fetched records is the
+ * paper's policy (Sec. 3.2); FIFO and RANDOM are the alternatives its cache study replays (Sec. 4.3, Fig. 6):
+ * FIFO - a hit does not refresh its slot (stamps record fetches only); victims are still the non-hit slots in
+ * ascending (stamp, slot) order.  RANDOM - recency is kept as for LRU but victims are the m non-hit slots with the
+ * smallest (key, slot), key = low 32 bits of mix64(mix64(seed ^ (r << 32 | group)) + (t << 32 | slot)), and the
+ * i-th miss takes the i-th victim in ascending slot order. */
+#define HISPARSE_POLICY_LRU 0
+#define HISPARSE_POLICY_FIFO 1
+#define HISPARSE_POLICY_RANDOM 2
+
 /* limits */
 #define HISPARSE_MAX_CACHE_SLOTS 16384
 #define HISPARSE_MAX_TOP_K 4096
@@ -89,6 +99,8 @@ typedef struct {
   uint32_t flags;            /* HISPARSE_FLAG_*                                                         */
   int32_t ctas_per_request;  /* thread blocks (one cluster) that share one request's fetch work;
                                 0 = choose from N (about 32 blocks in all); otherwise 1, 2, 4 or 8             */
+  int32_t policy;            /* HISPARSE_POLICY_*; 0 = the paper's LRU                                  */
+  uint64_t policy_seed;      /* RANDOM policy only                                                     */
 } hisparse_config_t;
 
 /* Sec. 3.3 step (2) "Admission": reserve the per-layer caches and metadata of N requests.  All

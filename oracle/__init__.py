@@ -3,4 +3,4 @@
 Only `tests/`, the smoke check and the benchmark's CPU-baseline / reference leg may import this
 package.  It shares no code with the CUDA library and never imports it.
 """
-from .oracle import Oracle, build, STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, FLAG_NO_BYTES, kv_footprint_bytes  # noqa: F401
+from .oracle import Oracle, build, STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, FLAG_NO_BYTES, kv_footprint_bytes, POLICY_LRU, POLICY_FIFO, POLICY_RANDOM  # noqa: F401

@@ -45,6 +45,17 @@
 #define ORACLE_STATUS_DUPLICATE 2u
 #define ORACLE_FLAG_NO_BYTES 1u /* metadata only: no cache pool, no record copies */
 
+/* Replacement policies.  LRU with hits above misses is the paper's policy (Sec. 3.2); FIFO and RANDOM are the
+ * alternatives its cache-locality study replays against the same selection stream (Sec. 4.3, Fig. 6):
+ *   FIFO   - a hit does not refresh a slot: stamps record the fetch only, victims are the non-hit slots in
+ *            ascending (fetch stamp, slot) order, i-th miss <-> i-th victim;
+ *   RANDOM - recency is kept as for LRU but not used for eviction: every non-hit slot gets the key
+ *            low32(mix64(mix64(seed ^ (r << 32 | group)) + (t << 32 | slot))), the m smallest (key, slot) are the
+ *            victims, and the i-th miss takes the i-th victim in ascending SLOT order. */
+#define ORACLE_POLICY_LRU 0
+#define ORACLE_POLICY_FIFO 1
+#define ORACLE_POLICY_RANDOM 2
+
 typedef struct {
   int N, L, lpg, G, B, k;
   int64_t E;
@@ -63,6 +74,9 @@ typedef struct {
   uint8_t **pool;                /* [L] -> [N][B+1][E] */
   uint8_t *replayed;             /* [L] plan replayed into this shared layer since the anchor ran */
   uint32_t status;
+  int policy;                    /* ORACLE_POLICY_* */
+  uint64_t policy_seed;          /* RANDOM only */
+  uint8_t *hit_flag;             /* [B] scratch: slot was hit in the current resolve */
 } oracle_t;
 
 static uint8_t *rec_host(oracle_t *o, int r, int l, int64_t p) {
@@ -112,7 +126,15 @@ oracle_t *oracle_create(int N, int L, int lpg, int B, int k, int64_t E, const in
   if (!(flags & ORACLE_FLAG_NO_BYTES))
     for (int l = 0; l < L; ++l) o->pool[l] = (uint8_t *)calloc((size_t)N * (B + 1), (size_t)E);
   o->replayed = (uint8_t *)calloc(L, 1);
+  o->hit_flag = (uint8_t *)calloc(B, 1);
   return o;
+}
+
+int oracle_set_policy(oracle_t *o, int policy, uint64_t seed) {
+  if (policy < ORACLE_POLICY_LRU || policy > ORACLE_POLICY_RANDOM) return -1;
+  o->policy = policy;
+  o->policy_seed = seed;
+  return 0;
 }
 
 void oracle_destroy(oracle_t *o) {
@@ -126,7 +148,7 @@ void oracle_destroy(oracle_t *o) {
   free(o->slot_pos); free(o->last_use); free(o->pos2slot); free(o->first_j); free(o->plan_pos);
   free(o->plan_slot); free(o->anchor_out); free(o->t); free(o->plan_n); free(o->anchor_hits);
   free(o->anchor_misses); free(o->pool); free(o->replayed); free(o->cap); free(o->len);
-  free(o->newest); free(o->host); free(o);
+  free(o->newest); free(o->host); free(o->hit_flag); free(o);
 }
 
 /* Sec. 3.3 step (4): every request appends one record per layer.  The record goes into the
@@ -147,7 +169,22 @@ int oracle_append(oracle_t *o, const uint8_t *new_kv /* [N][L][E] */) {
   return 0;
 }
 
+static uint64_t oracle_mix64(uint64_t z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+static uint32_t random_key(uint64_t seed, int r, int g, uint32_t t, int slot) {
+  uint64_t a = oracle_mix64(seed ^ (((uint64_t)(uint32_t)r << 32) | (uint32_t)g));
+  return (uint32_t)oracle_mix64(a + (((uint64_t)t << 32) | (uint32_t)slot));
+}
+
 typedef struct { uint32_t stamp; int32_t slot; } cand_t;
+static int cmp_slot(const void *a, const void *b) {
+  const cand_t *x = (const cand_t *)a, *y = (const cand_t *)b;
+  return (x->slot > y->slot) - (x->slot < y->slot);
+}
 static int cmp_cand(const void *a, const void *b) {
   const cand_t *x = (const cand_t *)a, *y = (const cand_t *)b;
   if (x->stamp != y->stamp) return x->stamp < y->stamp ? -1 : 1;
@@ -216,15 +253,21 @@ int oracle_resolve(oracle_t *o, int layer, const int32_t *sel, int32_t *slot_tab
       first_j[p] = j;
       if (p == o->newest[r]) { out[j] = B; ++h; continue; }   /* reserved newest-token slot */
       int32_t s = pos2slot[p];
-      if (s >= 0) { out[j] = s; last_use[s] = hit_stamp; ++h; }
+      if (s >= 0) { out[j] = s; o->hit_flag[s] = 1; if (o->policy != ORACLE_POLICY_FIFO) last_use[s] = hit_stamp; ++h; }
       else miss_j[m++] = j;
     }
 
     /* pass 2: eviction candidates = slots not hit in this resolve, ascending (stamp, slot) */
     int nc = 0;
     for (int s = 0; s < B; ++s)
-      if (last_use[s] != hit_stamp) { cand[nc].stamp = last_use[s]; cand[nc].slot = s; ++nc; }
+      if (!o->hit_flag[s]) {
+        cand[nc].stamp = o->policy == ORACLE_POLICY_RANDOM ? random_key(o->policy_seed, r, g, t, s) : last_use[s];
+        cand[nc].slot = s;
+        ++nc;
+      }
     qsort(cand, (size_t)nc, sizeof(cand_t), cmp_cand);
+    if (o->policy == ORACLE_POLICY_RANDOM) qsort(cand, (size_t)(m < nc ? m : nc), sizeof(cand_t), cmp_slot);
+    memset(o->hit_flag, 0, (size_t)B);
 
     /* pass 3: the i-th miss (selection order) takes the i-th candidate */
     for (int q = 0; q < m; ++q) {

@@ -19,6 +19,7 @@ _SO = os.path.join(_HERE, "_hisparse_oracle.so")
 STATUS_OUT_OF_RANGE = 1
 STATUS_DUPLICATE = 2
 FLAG_NO_BYTES = 1
+POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -64,6 +65,8 @@ def _L() -> ctypes.CDLL:
         L.oracle_status.restype = u32
         L.oracle_clear_status.argtypes = [vp]
         L.oracle_clear_status.restype = None
+        L.oracle_set_policy.argtypes = [vp, i32, ctypes.c_uint64]
+        L.oracle_set_policy.restype = i32
         L.oracle_kv_footprint_bytes.argtypes = [i64, i64, i64, i64]
         L.oracle_kv_footprint_bytes.restype = i64
         _lib = L
@@ -89,7 +92,8 @@ class Oracle:
 
     def __init__(self, num_requests: int, num_layers: int, layers_per_group: int, cache_slots: int,
                  top_k: int, entry_bytes: int, capacity: Sequence[int], init_len: Sequence[int],
-                 host_history: Sequence[np.ndarray] | None = None, flags: int = 0):
+                 host_history: Sequence[np.ndarray] | None = None, flags: int = 0, policy: int = POLICY_LRU,
+                 policy_seed: int = 0):
         self.N, self.L, self.lpg, self.B, self.k, self.E = (num_requests, num_layers, layers_per_group,
                                                             cache_slots, top_k, entry_bytes)
         self.capacity = np.asarray(capacity, dtype=np.int64)
@@ -109,6 +113,9 @@ class Oracle:
         if not self._h:
             raise ValueError("oracle_create rejected the configuration")
         self.flags = flags
+        if _L().oracle_set_policy(self._h, policy, policy_seed) != 0:
+            raise ValueError("unknown replacement policy")
+        self.policy = policy
 
     def close(self):
         if getattr(self, "_h", None):

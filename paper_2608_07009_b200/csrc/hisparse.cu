@@ -74,6 +74,8 @@ struct DevState {
   int io_threads, io_depth, io_chunk;  // fetch pipeline: issuing threads, ring slots per thread, bytes per piece
   int ring_bytes;                  // io_threads * io_depth * io_chunk
   int io_ppr;                      // pieces per record = ceil(E / io_chunk)
+  int policy;                      // HISPARSE_POLICY_*
+  unsigned long long policy_seed;  // RANDOM policy
   unsigned long long *phase_ns;    // [N][16]: 8 globaltimer stamps, then 8 SM cycle-counter stamps (PHASE_TIMERS)
 };
 
@@ -315,6 +317,85 @@ __device__ __forceinline__ void table_lookup(const unsigned long long *tab, cons
   }
 }
 
+
+// Key of the RANDOM replacement policy for one slot at resolve t of (request r, group g): the low 32 bits of
+// mix64(mix64(seed ^ (r << 32 | g)) + (t << 32 | slot)), mix64 being the splitmix64 finaliser after adding its
+// golden-ratio increment.  Victims are the m candidate slots with the smallest (key, slot).
+__device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
+  z += 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+__device__ __forceinline__ uint32_t random_key(unsigned long long base, uint32_t t, int slot) {
+  return (uint32_t)mix64(base + (((unsigned long long)t << 32) | (uint32_t)slot));
+}
+
+// RANDOM policy: marks in s_vicbits the m slots without a hit bit that have the smallest (key, slot).
+// Radix select, most significant byte first, with a 256-bin histogram in shared memory (s_hist: 257 ints).
+template <int IPT>
+__device__ __forceinline__ void select_random_victims(const int B, const int m, const unsigned long long base,
+                                                      const uint32_t t, const uint32_t *s_hitbits, uint32_t *s_vicbits,
+                                                      int *s_hist, int *s_warp) {
+  const int tid = threadIdx.x;
+  if (m == 0) return;
+  uint32_t key[IPT];
+  uint32_t cand = 0;  // this thread owns slots tid*IPT .. tid*IPT+IPT-1 (consecutive: ties are broken by slot)
+#pragma unroll
+  for (int i = 0; i < IPT; ++i) {
+    const int s = tid * IPT + i;
+    key[i] = 0;
+    if (s < B && !((s_hitbits[s >> 5] >> (s & 31)) & 1u)) {
+      cand |= 1u << i;
+      key[i] = random_key(base, t, s);
+    }
+  }
+  uint32_t prefix = 0;
+  int remaining = m;
+#pragma unroll 1
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 257; i += blockDim.x) s_hist[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < IPT; ++i)
+      if (((cand >> i) & 1u) && (shift == 24 || (key[i] >> (shift + 8)) == prefix))
+        atomicAdd(&s_hist[(key[i] >> shift) & 255u], 1);
+    __syncthreads();
+    if (tid == 0) {  // the byte at which the running count reaches `remaining`
+      int acc = 0, b = 0;
+      for (; b < 255; ++b) {
+        if (acc + s_hist[b] >= remaining) break;
+        acc += s_hist[b];
+      }
+      s_hist[256] = (b << 16) | acc;  // acc < 2^15 (at most B candidates)
+    }
+    __syncthreads();
+    const int packed = s_hist[256];
+    prefix = (prefix << 8) | (uint32_t)(packed >> 16);
+    remaining -= packed & 0xffff;
+    __syncthreads();
+  }
+  // keys below the threshold are victims; of the keys equal to it, the first `remaining` in slot order
+  uint32_t eq = 0;
+#pragma unroll
+  for (int i = 0; i < IPT; ++i)
+    if ((cand >> i) & 1u) {
+      const int s = tid * IPT + i;
+      if (key[i] < prefix) atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
+      else if (key[i] == prefix) eq |= 1u << i;
+    }
+  int total;
+  int rank = block_scan_excl(__popc(eq), s_warp, total);
+#pragma unroll
+  for (int i = 0; i < IPT; ++i)
+    if ((eq >> i) & 1u) {
+      const int s = tid * IPT + i;
+      if (rank < remaining) atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
+      ++rank;
+    }
+  __syncthreads();
+}
+
 // Everything the first block of a cluster does before the fetch can start: Phases 1-3 of Sec. 3.4.
 // IPT = entries of the recency order per thread (B <= IPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
 // the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
@@ -326,8 +407,9 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  uint32_t *s_vicbits, uint16_t *s_order, int *s_warp, int *s_misc,
                                                  const int64_t cap_r, const int64_t init_len_r,
                                                  const int64_t p2s_off_r, unsigned long long *stamps,
-                                                 unsigned char *s_ring, unsigned long long *s_bars, int &m,
-                                                 int &n_nonhit, uint32_t &my_status) {
+                                                 unsigned char *s_ring, unsigned long long *s_bars,
+                                                 const uint32_t t_now, int *s_warp_pre, int &m, int &n_nonhit,
+                                                 uint32_t &my_status) {
   constexpr int T = kThreads;
   const int tid = threadIdx.x;
   const int k = d.k, B = d.B, H = d.H;
@@ -464,22 +546,76 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     m = total & 0xffff;
     n_nonhit = total >> 16;
     int mrank = excl & 0xffff, nrank = excl >> 16;
-    // the i-th miss (selection order) takes the i-th non-hit slot of the recency order
 #pragma unroll
     for (int i = 0; i < kSelPerThread; ++i)
       if ((miss_mask >> i) & 1u) s_plan_pos[mrank++] = tid * kSelPerThread + i;
+    if (d.policy == HISPARSE_POLICY_LRU) {
+      // the i-th miss (selection order) takes the i-th non-hit slot of the recency order
 #pragma unroll
-    for (int i = 0; i < IPT; ++i)
-      if ((nh_mask >> i) & 1u) {
+      for (int i = 0; i < IPT; ++i)
+        if ((nh_mask >> i) & 1u) {
+          const int s = slot[i];
+          if (nrank < m) {
+            s_plan_slot[nrank] = s;
+            atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
+          } else {
+            s_order[nrank - m] = (uint16_t)s;  // in place: every thread read its entries before the scan's barriers
+          }
+          ++nrank;
+        }
+    } else if (d.policy == HISPARSE_POLICY_FIFO) {
+      // same victims, but a hit does not move: everything that is not a victim keeps its place in the list
+#pragma unroll
+      for (int i = 0; i < IPT; ++i) {
+        const int q = tid * IPT + i;
+        if (q >= B) break;
         const int s = slot[i];
-        if (nrank < m) {
+        const bool nonhit = (nh_mask >> i) & 1u;
+        if (nonhit && nrank < m) {
           s_plan_slot[nrank] = s;
           atomicOr(&s_vicbits[s >> 5], 1u << (s & 31));
         } else {
-          s_order[nrank - m] = (uint16_t)s;  // in place: every thread read its entries before the scan's barriers
+          s_order[q - (nrank < m ? nrank : m)] = (uint16_t)s;
         }
-        ++nrank;
+        if (nonhit) ++nrank;
       }
+    } else {
+      // RANDOM: victims by hashed key, paired with the misses in ascending slot order; the list is kept as for LRU
+      __syncthreads();
+      const unsigned long long base = mix64(d.policy_seed ^ (((unsigned long long)(uint32_t)r << 32) | (uint32_t)(rg - (int64_t)r * d.G)));
+      select_random_victims<IPT>(B, m, base, t_now, s_hitbits, s_vicbits, reinterpret_cast<int *>(s_tab), s_warp);
+      uint32_t keep = 0;
+#pragma unroll
+      for (int i = 0; i < IPT; ++i)
+        if (((nh_mask >> i) & 1u) && !((s_vicbits[slot[i] >> 5] >> (slot[i] & 31)) & 1u)) keep |= 1u << i;
+      int tot2;
+      int krank = block_scan_excl(__popc(keep), s_warp, tot2);
+#pragma unroll
+      for (int i = 0; i < IPT; ++i)
+        if ((keep >> i) & 1u) s_order[krank++] = (uint16_t)slot[i];
+      // i-th victim in slot order: running count of victim bits below each word, by warp 0
+      if (tid < 32) {
+        int run = 0;
+        for (int wb = 0; wb < d.W; wb += 32) {
+          const int w = wb + tid;
+          const int c = w < d.W ? __popc(s_vicbits[w]) : 0;
+          int inc = c;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (tid >= o) inc += n;
+          }
+          if (w < d.W) s_warp_pre[w] = run + inc - c;
+          run += __shfl_sync(0xffffffffu, inc, 31);
+        }
+      }
+      __syncthreads();
+      for (int s = tid; s < B; s += T) {
+        const uint32_t vw = s_vicbits[s >> 5], bit = 1u << (s & 31);
+        const int i = s_warp_pre[s >> 5] + __popc(vw & (bit - 1u));
+        if ((vw & bit) && i < m) s_plan_slot[i] = s;
+      }
+    }
   }
   if (timers && tid == 0) stamps[13] = clock64();
   __syncthreads();
@@ -541,7 +677,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     const int32_t *row = sel + (int64_t)r * k;
 #define HS_META(IPT)                                                                                              \
   resolve_metadata<IPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits, s_order, \
-                        s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, m, n_nonhit, my_status)
+                        s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t, s_vicpre, m, n_nonhit, my_status)
     if (B <= 4 * T) HS_META(4);
     else if (B <= 8 * T) HS_META(8);
     else HS_META(16);
@@ -605,17 +741,26 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
     }
     __syncthreads();
-    const int n_surv = n_nonhit - m;
     uint32_t *last_use = d.last_use + rg * B;
-    for (int s = tid; s < B; s += T) {
-      const int w = s >> 5;
-      const uint32_t bit = 1u << (s & 31), lt = bit - 1u;
-      const uint32_t vw = s_vicbits[w], hw = s_hitbits[w];
-      if (vw & bit) {
-        s_order[n_surv + s_vicpre[w] + __popc(vw & lt)] = (uint16_t)s;
-      } else if (hw & bit) {
-        s_order[n_nonhit + s_hitpre[w] + __popc(hw & lt)] = (uint16_t)s;
-        last_use[s] = 2u * t + 1u;  // hits are stamped above this step's fetched records
+    if (d.policy == HISPARSE_POLICY_FIFO) {
+      // insertion order: the refilled slots go to the end, by slot; hits were left where they were, unstamped
+      for (int s = tid; s < B; s += T) {
+        const int w = s >> 5;
+        const uint32_t bit = 1u << (s & 31), vw = s_vicbits[w];
+        if (vw & bit) s_order[(B - m) + s_vicpre[w] + __popc(vw & (bit - 1u))] = (uint16_t)s;
+      }
+    } else {
+      const int n_surv = n_nonhit - m;
+      for (int s = tid; s < B; s += T) {
+        const int w = s >> 5;
+        const uint32_t bit = 1u << (s & 31), lt = bit - 1u;
+        const uint32_t vw = s_vicbits[w], hw = s_hitbits[w];
+        if (vw & bit) {
+          s_order[n_surv + s_vicpre[w] + __popc(vw & lt)] = (uint16_t)s;
+        } else if (hw & bit) {
+          s_order[n_nonhit + s_hitpre[w] + __popc(hw & lt)] = (uint16_t)s;
+          last_use[s] = 2u * t + 1u;  // hits are stamped above this step's fetched records
+        }
       }
     }
     __syncthreads();
@@ -905,11 +1050,12 @@ int validate_config(const hisparse_config_t *c) {
   }
   const int s = c->ctas_per_request;
   if (!(s == 0 || s == 1 || s == 2 || s == 4 || s == 8)) return HISPARSE_EINVAL;
+  if (c->policy < HISPARSE_POLICY_LRU || c->policy > HISPARSE_POLICY_RANDOM) return HISPARSE_EINVAL;
   return HISPARSE_OK;
 }
 
 int hash_size(int k) {
-  int H = 32;
+  int H = 256;  // never below 2 KB: the RANDOM policy reuses the table's memory for a 257-word histogram
   while (H < 2 * k) H <<= 1;
   return H;
 }
@@ -1014,6 +1160,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   d.hshift = 32;
   for (int x = d.H; x > 1; x >>= 1) --d.hshift;
   d.E = c->entry_bytes; d.upe = (uint32_t)(c->entry_bytes / 16); d.flags = c->flags;
+  d.policy = c->policy; d.policy_seed = c->policy_seed;
   d.layer_pool_bytes = (int64_t)N * (B + 1) * d.E;
   h->cap.assign(c->capacity, c->capacity + N);
   h->init_len.assign(c->init_len, c->init_len + N);

@@ -19,6 +19,7 @@ NOALLOC_MAX_REQUESTS, NOALLOC_MAX_SELECTIONS = 1024, 65536
 FLAG_SKIP_IO, FLAG_DEBUG_VALIDATE, FLAG_INLINE_WRITE_THROUGH, FLAG_PHASE_TIMERS, FLAG_NO_PDL = 1, 2, 4, 8, 16
 STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, STATUS_CAPACITY, STATUS_INCONSISTENT, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 MAX_CACHE_SLOTS, MAX_TOP_K = 16384, 4096
+POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2
 
 EXPORTS = [
     "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch",
@@ -44,6 +45,7 @@ class Config(ctypes.Structure):
         ("cache_slots", ctypes.c_int32), ("top_k", ctypes.c_int32), ("entry_bytes", ctypes.c_int64),
         ("capacity", ctypes.c_void_p), ("init_len", ctypes.c_void_p), ("host_history", ctypes.c_void_p),
         ("device", ctypes.c_int32), ("flags", ctypes.c_uint32), ("ctas_per_request", ctypes.c_int32),
+        ("policy", ctypes.c_int32), ("policy_seed", ctypes.c_uint64),
     ]
 
 
@@ -152,7 +154,7 @@ def device_bytes(num_requests, num_layers, layers_per_group, cache_slots, top_k,
     cap = np.asarray(capacity, dtype=np.int64)
     il = np.zeros_like(cap)
     cfg = Config(num_requests, num_layers, layers_per_group, cache_slots, top_k, entry_bytes,
-                 cap.ctypes.data, il.ctypes.data, None, 0, 0, 0)
+                 cap.ctypes.data, il.ctypes.data, None, 0, 0, 0, 0, 0)
     kv, meta = ctypes.c_size_t(), ctypes.c_size_t()
     _check(lib().hisparse_device_bytes(ctypes.byref(cfg), ctypes.byref(kv), ctypes.byref(meta)), "hisparse_device_bytes")
     return kv.value, meta.value
@@ -193,7 +195,7 @@ class HiSparse:
 
     def __init__(self, num_requests: int, num_layers: int, layers_per_group: int, cache_slots: int, top_k: int,
                  entry_bytes: int, capacity: Sequence[int], init_len: Sequence[int], host_history: Sequence,
-                 device: int = 0, flags: int = 0, ctas_per_request: int = 0):
+                 device: int = 0, flags: int = 0, ctas_per_request: int = 0, policy: int = 0, policy_seed: int = 0):
         self.N, self.L, self.lpg, self.B, self.k, self.E = (num_requests, num_layers, layers_per_group, cache_slots,
                                                             top_k, entry_bytes)
         self.device = device
@@ -205,7 +207,7 @@ class HiSparse:
         ptrs = (ctypes.c_void_p * num_requests)(*[h.ptr if isinstance(h, HostHistory) else int(h) for h in host_history])
         cfg = Config(num_requests, num_layers, layers_per_group, cache_slots, top_k, entry_bytes,
                      self.capacity.ctypes.data, self.init_len.ctypes.data, ctypes.addressof(ptrs), device, flags,
-                     ctas_per_request)
+                     ctas_per_request, policy, policy_seed)
         h = ctypes.c_void_p()
         _check(lib().hisparse_create(ctypes.byref(cfg), ctypes.byref(h)), "hisparse_create")
         self._h = h

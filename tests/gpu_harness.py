@@ -13,7 +13,7 @@ class Pair:
     """One CUDA handle and one oracle over separate copies of the same host histories."""
 
     def __init__(self, w: inputs.Workload, flags: int = 0, ctas_per_request: int = 0, oracle_bytes: bool = True,
-                 device: int = 0):
+                 device: int = 0, policy: int = 0, policy_seed: int = 0):
         self.w = w
         self.dev = torch.device("cuda:%d" % device)
         cap, il = w.capacity, w.init_len
@@ -21,16 +21,17 @@ class Pair:
         for r, h in enumerate(self.hist_gpu):
             inputs.fill_history(h.ptr, r, w.num_layers, cap[r], 0, il[r], w.entry_bytes, w.seed)
         self.gpu = HiSparse(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k, w.entry_bytes,
-                            cap, il, self.hist_gpu, device=device, flags=flags, ctas_per_request=ctas_per_request)
+                            cap, il, self.hist_gpu, device=device, flags=flags, ctas_per_request=ctas_per_request,
+                            policy=policy, policy_seed=policy_seed)
         self.oracle_bytes = oracle_bytes
         if oracle_bytes:
             self.hist_cpu = [inputs.new_history(w, r) for r in range(w.num_requests)]
             self.oracle = Oracle(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k,
-                                 w.entry_bytes, cap, il, self.hist_cpu)
+                                 w.entry_bytes, cap, il, self.hist_cpu, policy=policy, policy_seed=policy_seed)
         else:
             self.hist_cpu = None
             self.oracle = Oracle(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k,
-                                 w.entry_bytes, cap, il, None, FLAG_NO_BYTES)
+                                 w.entry_bytes, cap, il, None, FLAG_NO_BYTES, policy=policy, policy_seed=policy_seed)
         self.mism = torch.zeros(1, dtype=torch.int32, device=self.dev)
 
     def close(self):
@@ -112,9 +113,10 @@ class Pair:
 
 
 def run_trace(w: inputs.Workload, steps: int, flags: int = 0, ctas_per_request: int = 0, oracle_bytes: bool = True,
-              state_every: int = 1, pool_every: int = 0, use_prefetch: bool = False, state_requests=None):
+              state_every: int = 1, pool_every: int = 0, use_prefetch: bool = False, state_requests=None,
+              policy: int = 0, policy_seed: int = 0):
     """Replays `steps` steps of the workload's trace through both sides, comparing as it goes."""
-    pair = Pair(w, flags, ctas_per_request, oracle_bytes)
+    pair = Pair(w, flags, ctas_per_request, oracle_bytes, policy=policy, policy_seed=policy_seed)
     side = torch.cuda.Stream() if use_prefetch else None
     tr = inputs.Trace(w)
     total_h = total_m = 0

@@ -12,8 +12,30 @@ from __future__ import annotations
 from typing import List, Sequence
 
 
+MASK64 = (1 << 64) - 1
+
+
+def mix64(z: int) -> int:
+    z = (z + 0x9E3779B97F4A7C15) & MASK64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & MASK64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & MASK64
+    return z ^ (z >> 31)
+
+
+def random_key(seed: int, r: int, g: int, t: int, slot: int) -> int:
+    """Key of the RANDOM policy: low 32 bits of mix64(mix64(seed ^ (r << 32 | g)) + (t << 32 | slot))."""
+    a = mix64(seed ^ ((r << 32) | g))
+    return mix64((a + ((t << 32) | slot)) & MASK64) & 0xFFFFFFFF
+
+
 class ListLRUSim:
-    def __init__(self, cache_slots: int, top_k: int, length: int):
+    """policy: "lru" (hits to the most-recent end), "fifo" (hits leave the list alone: insertion order) or
+    "random" (list kept as for lru; victims = the m non-hit slots with the smallest hashed key, paired with the
+    misses in ascending slot order)."""
+
+    def __init__(self, cache_slots: int, top_k: int, length: int, policy: str = "lru", seed: int = 0,
+                 request: int = 0, group: int = 0):
+        self.policy, self.seed, self.request, self.group, self.t = policy, seed, request, group, 0
         self.B, self.k = cache_slots, top_k
         self.order: List[int] = list(range(cache_slots))  # least recent first
         self.slot_pos: List[int] = [-1] * cache_slots
@@ -56,15 +78,23 @@ class ListLRUSim:
                 hits += 1
             else:
                 miss_js.append(j)
+        self.t += 1
         not_hit = [s for s in self.order if s not in hit_slots]
-        victims = not_hit[: len(miss_js)]
-        untouched = not_hit[len(miss_js):]
+        if self.policy == "random":
+            ranked = sorted(not_hit, key=lambda s: (random_key(self.seed, self.request, self.group, self.t, s), s))
+            victims = sorted(ranked[: len(miss_js)])
+        else:
+            victims = not_hit[: len(miss_js)]
         evicted = []
         for j, v in zip(miss_js, victims):
             evicted.append(self.slot_pos[v])
             self.slot_pos[v] = int(row[j])
             out[j] = v
-        self.order = untouched + sorted(victims) + sorted(hit_slots)
+        if self.policy == "fifo":
+            self.order = [s for s in self.order if s not in victims] + sorted(victims)
+        else:
+            untouched = [s for s in not_hit if s not in victims]
+            self.order = untouched + sorted(victims) + sorted(hit_slots)
         for j, j0 in follows.items():
             out[j] = out[j0]
         plan = [(int(row[j]), v) for j, v in zip(miss_js, victims)]

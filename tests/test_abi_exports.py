@@ -43,7 +43,7 @@ def test_create_validates_before_touching_a_device():
     from paper_2608_07009_b200 import hisparse as hs
     cap = np.array([64], dtype=np.int64)
     il = np.array([10], dtype=np.int64)
-    cfg = hs.Config(1, 1, 1, 4, 8, 32, cap.ctypes.data, il.ctypes.data, None, 0, 0, 0)    # k > B
+    cfg = hs.Config(1, 1, 1, 4, 8, 32, cap.ctypes.data, il.ctypes.data, None, 0, 0, 0, 0, 0)    # k > B
     h = ctypes.c_void_p()
     assert hs.lib().hisparse_create(ctypes.byref(cfg), ctypes.byref(h)) == hs.EINVAL
     assert not h.value

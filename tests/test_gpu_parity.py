@@ -196,6 +196,37 @@ def test_skip_io_keeps_metadata_exact():
         pair.close()
 
 
+# ------------------------------------------------------------------ replacement policies of the ablation
+
+@pytest.mark.parametrize("policy", [hs.POLICY_FIFO, hs.POLICY_RANDOM])
+def test_policies_tiny(policy):
+    rng = np.random.default_rng(policy)
+    for B, k in ((1, 1), (3, 2), (8, 8), (12, 5), (40, 17)):
+        w = tiny_workload(2, 1, 1, k, B, 48, [3 * B + 2, 2 * B + 1])
+        pair = Pair(w, policy=policy, policy_seed=99, flags=hs.FLAG_DEBUG_VALIDATE)
+        try:
+            for step in range(40):
+                if step % 5 == 4:
+                    pair.append()
+                rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0] for r in range(2)])
+                pair.resolve_and_compare(0, rows)
+                pair.compare_state(0)
+            pair.finish()
+        finally:
+            pair.close()
+
+
+@pytest.mark.parametrize("policy", [hs.POLICY_FIFO, hs.POLICY_RANDOM])
+def test_policies_c2_shape_and_groups(policy):
+    w = inputs.c2_dsa_decode(num_requests=3, num_layers=2, steps=6, context=6000)
+    run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=7)
+    w = inputs.c3_dsa_long(0.5, steps=4, short_ctx=5000, long_ctx=40000, num_short=2)
+    run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=7, use_prefetch=True)
+    w = inputs.Workload("ragged", inputs.KIND_DSA_MIX, 2, 1, 1, 1000, 9001, 32, [12000, 9500], 5,
+                        keep=700, recent_window=300, seed=3, config_id=9)
+    run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=7)
+
+
 # ------------------------------------------------------------------ CUDA graph replay of whole steps
 
 def test_graph_replay_matches_oracle():
