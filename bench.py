@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--no-prefetch", action="store_true", help="c3 only: shared layers swap in synchronously")
     ap.add_argument("--skip-io", action="store_true", help="no-IO timing mode (metadata only)")
     ap.add_argument("--phases", action="store_true", help="record the resolve kernel's phase stamps (adds a little time)")
+    ap.add_argument("--spec-hint", action="store_true",
+                    help="speculative prefetch: layer l's selection is given to layer l+1 as a hint (side stream)")
     ap.add_argument("--no-pdl", action="store_true", help="launch Resolve without programmatic dependent launch")
     ap.add_argument("--no-all-hit", action="store_true", help="skip the scaled all-hit HBM point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -280,7 +282,9 @@ def run_ours(args):
         raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    launched = "WORLD_SIZE" in os.environ          # under torchrun, also with a single rank
+    if launched:
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")   # keep stdout to the one JSON line
         dist.init_process_group("nccl", device_id=dev)
 
     w = make_workload(args, rank)
@@ -342,6 +346,9 @@ def run_ours(args):
             if ev is not None:
                 ev[layer][1].record(stream)
             n += 1 if layer % lpg == 0 or use_prefetch else 2
+            if args.spec_hint and lpg == 1 and layer + 1 < L:
+                gpu.prefetch_hint(layer + 1, sel_st[layer], side, stream=stream)
+                n += 1
             if use_prefetch and layer % lpg == 0:
                 for l2 in range(layer + 1, layer + lpg):
                     gpu.prefetch(l2, side)
@@ -350,7 +357,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
+        if launched:
             dist.barrier()
             torch.cuda.synchronize()
 
@@ -487,7 +494,7 @@ def run_ours(args):
             "value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": "requests 0..%d of %d, all %d layers, %d steps after the cold step and 1 warm-up step" % (
                 n_req - 1, N, L, steps_cpu)}
-    if world > 1:
+    if launched:
         dist.barrier()
         dist.destroy_process_group()
     if rank != 0:

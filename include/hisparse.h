@@ -150,6 +150,15 @@ int hisparse_resolve(hisparse_t *h, int layer, const int32_t *sel_dev, int32_t *
  * been resolved in this step (ESTATE otherwise).  The later hisparse_resolve(layer) waits for it. */
 int hisparse_prefetch(hisparse_t *h, int layer, void *side_stream);
 
+/* Sec. 3.5 "A speculative alternative": for models WITHOUT shared selections, use some other selection (the
+ * paper: the previous layer's) as a hint for `layer` and bring the hinted records in ahead of the layer's own
+ * resolve.  Defined here as exactly a resolve of `layer` with hint_sel_dev [N][k] as its selection, run on
+ * side_stream after the work already enqueued on `stream`, with its slot table and counts discarded: hinted
+ * records that were host-only are fetched (evicting LRU victims) and the hinted positions are stamped.  A wrong
+ * hint costs transfers and cache space, never correctness: the layer's own hisparse_resolve, which waits for the
+ * hint, still finds or fetches every selected record.  Only with layers_per_group == 1 (EINVAL otherwise). */
+int hisparse_prefetch_hint(hisparse_t *h, int layer, const int32_t *hint_sel_dev, void *stream, void *side_stream);
+
 /* Makes `stream` wait for everything the library has in flight on its own backup stream and on
  * side streams given to hisparse_prefetch.  Needed before ending a stream capture that contains an
  * append, and before the host reads the histories.  The resolve of the last layer joins the

@@ -1022,6 +1022,11 @@ struct hisparse {
   std::vector<uint8_t> anchor_done;   // [G] the anchor has been resolved at least once
   std::vector<uint8_t> replayed;      // [L] plan replayed (or being replayed) since the anchor's last resolve
   std::vector<uint8_t> pref_unjoined; // [L] a side-stream replay that no stream has waited for yet
+  // speculative hints (hisparse_prefetch_hint): discarded outputs, fork / completion events
+  int32_t *hint_table = nullptr, *hint_hits = nullptr, *hint_misses = nullptr;
+  cudaEvent_t ev_hint_fork = nullptr;
+  std::vector<cudaEvent_t> ev_hint;   // [L]
+  std::vector<uint8_t> hint_unjoined; // [L]
 };
 
 namespace {
@@ -1232,6 +1237,9 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRY(dev_alloc(h, &d.n_appends, 1));
   HS_TRY(dev_alloc(h, &d.ticket, 1));
   HS_TRY(dev_alloc(h, &d.status, 1));
+  HS_TRY(dev_alloc(h, &h->hint_table, (size_t)N * k));
+  HS_TRY(dev_alloc(h, &h->hint_hits, (size_t)N));
+  HS_TRY(dev_alloc(h, &h->hint_misses, (size_t)N));
   HS_TRY(dev_alloc(h, &d.phase_ns, (size_t)N * 16));
 #undef HS_TRY
   d.cap = h->d_cap; d.init_len = h->d_init_len; d.p2s_off = h->d_p2s_off; d.host = h->d_host;
@@ -1264,6 +1272,10 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   h->ev_pref.assign(L, nullptr);
   for (int g = 0; g < G; ++g) HS_TRYC(cudaEventCreateWithFlags(&h->ev_plan[g], cudaEventDisableTiming));
   for (int l = 0; l < L; ++l) HS_TRYC(cudaEventCreateWithFlags(&h->ev_pref[l], cudaEventDisableTiming));
+  HS_TRYC(cudaEventCreateWithFlags(&h->ev_hint_fork, cudaEventDisableTiming));
+  h->ev_hint.assign(L, nullptr);
+  for (int l = 0; l < L; ++l) HS_TRYC(cudaEventCreateWithFlags(&h->ev_hint[l], cudaEventDisableTiming));
+  h->hint_unjoined.assign(L, 0);
   h->anchor_done.assign(G, 0);
   h->replayed.assign(L, 0);
   h->pref_unjoined.assign(L, 0);
@@ -1279,6 +1291,8 @@ int hisparse_destroy(hisparse_t *h) {
   cudaDeviceSynchronize();
   for (cudaEvent_t e : h->ev_plan) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : h->ev_pref) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : h->ev_hint) if (e) cudaEventDestroy(e);
+  if (h->ev_hint_fork) cudaEventDestroy(h->ev_hint_fork);
   if (h->ev_fork) cudaEventDestroy(h->ev_fork);
   if (h->ev_wt) cudaEventDestroy(h->ev_wt);
   if (h->backup) cudaStreamDestroy(h->backup);
@@ -1294,11 +1308,16 @@ int hisparse_join(hisparse_t *h, void *stream) {
     HS_CUDA(cudaStreamWaitEvent(st, h->ev_wt, 0));
     h->wt_pending = false;
   }
-  for (int l = 0; l < h->d.L; ++l)
+  for (int l = 0; l < h->d.L; ++l) {
     if (h->pref_unjoined[l]) {
       HS_CUDA(cudaStreamWaitEvent(st, h->ev_pref[l], 0));
       h->pref_unjoined[l] = 0;
     }
+    if (h->hint_unjoined[l]) {
+      HS_CUDA(cudaStreamWaitEvent(st, h->ev_hint[l], 0));
+      h->hint_unjoined[l] = 0;
+    }
+  }
   return HISPARSE_OK;
 }
 
@@ -1331,6 +1350,10 @@ int hisparse_resolve(hisparse_t *h, int layer, const int32_t *sel_dev, int32_t *
   int rc = HISPARSE_OK;
   if (layer % lpg == 0) {
     if (!sel_dev) return HISPARSE_EINVAL;
+    if (h->hint_unjoined[layer]) {  // a speculative hint for this layer is still in flight on a side stream
+      HS_CUDA(cudaStreamWaitEvent(st, h->ev_hint[layer], 0));
+      h->hint_unjoined[layer] = 0;
+    }
     // replays of the previous plan of this group must be over before the plan is overwritten
     for (int l = layer + 1; l < layer + lpg; ++l)
       if (h->pref_unjoined[l]) {
@@ -1380,6 +1403,23 @@ int hisparse_prefetch(hisparse_t *h, int layer, void *side_stream) {
   HS_CUDA(cudaEventRecord(h->ev_pref[layer], st));
   h->replayed[layer] = 1;
   h->pref_unjoined[layer] = 1;
+  return HISPARSE_OK;
+}
+
+int hisparse_prefetch_hint(hisparse_t *h, int layer, const int32_t *hint_sel_dev, void *stream, void *side_stream) {
+  if (!h || layer < 0 || layer >= h->d.L || !hint_sel_dev) return HISPARSE_EINVAL;
+  if (h->d.lpg != 1) return HISPARSE_EINVAL;  // shared-selection groups use the exact prefetch instead
+  cudaStream_t st = as_stream(stream), side = as_stream(side_stream);
+  HS_CUDA(cudaEventRecord(h->ev_hint_fork, st));
+  HS_CUDA(cudaStreamWaitEvent(side, h->ev_hint_fork, 0));
+  if (h->hint_unjoined[layer]) {  // an earlier hint for the same layer: keep them in order
+    HS_CUDA(cudaStreamWaitEvent(side, h->ev_hint[layer], 0));
+  }
+  const int rc = launch_resolve(h, layer, hint_sel_dev, h->hint_table, h->hint_hits, h->hint_misses, side);
+  if (rc) return rc;
+  h->anchor_done[layer] = 1;
+  HS_CUDA(cudaEventRecord(h->ev_hint[layer], side));
+  h->hint_unjoined[layer] = 1;
   return HISPARSE_OK;
 }
 

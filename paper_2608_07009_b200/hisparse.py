@@ -22,7 +22,7 @@ MAX_CACHE_SLOTS, MAX_TOP_K = 16384, 4096
 POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2
 
 EXPORTS = [
-    "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch",
+    "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch", "hisparse_prefetch_hint",
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
     "hisparse_clear_status", "hisparse_dump_state", "hisparse_dump_plan", "hisparse_device_bytes",
     "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
@@ -80,6 +80,7 @@ def lib() -> ctypes.CDLL:
             "hisparse_append": ([vp, vp, vp], i32),
             "hisparse_resolve": ([vp, i32, vp, vp, vp, vp, vp], i32),
             "hisparse_prefetch": ([vp, i32, vp], i32),
+            "hisparse_prefetch_hint": ([vp, i32, vp, vp, vp], i32),
             "hisparse_join": ([vp, vp], i32),
             "hisparse_layer_pool": ([vp, i32], vp),
             "hisparse_gather": ([vp, i32, vp, vp, vp], i32),
@@ -245,6 +246,10 @@ class HiSparse:
 
     def prefetch(self, layer: int, side_stream) -> None:
         _check(lib().hisparse_prefetch(self._h, layer, _stream_ptr(side_stream)), "hisparse_prefetch")
+
+    def prefetch_hint(self, layer: int, hint_sel, side_stream, stream=None) -> None:
+        _check(lib().hisparse_prefetch_hint(self._h, layer, _dev_ptr(hint_sel, "int32", self.N * self.k),
+                                            _stream_ptr(stream), _stream_ptr(side_stream)), "hisparse_prefetch_hint")
 
     def join(self, stream=None) -> None:
         _check(lib().hisparse_join(self._h, _stream_ptr(stream)), "hisparse_join")

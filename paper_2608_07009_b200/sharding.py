@@ -21,7 +21,7 @@ def aggregate(elapsed_s: float, units: float, device=None) -> Tuple[float, float
     """(max over ranks of elapsed_s, sum over ranks of units); identity without a process group."""
     import torch
     import torch.distributed as dist
-    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+    if not (dist.is_available() and dist.is_initialized()):
         return float(elapsed_s), float(units)
     t = torch.tensor([elapsed_s], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)

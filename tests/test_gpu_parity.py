@@ -227,6 +227,39 @@ def test_policies_c2_shape_and_groups(policy):
     run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=7)
 
 
+# ------------------------------------------------------------------ speculative hints
+
+def test_speculative_hint_is_a_discarded_resolve():
+    # layer l's selection as a hint for layer l+1 (Sec. 3.5): on the oracle side a hint is one more resolve
+    w = inputs.c2_dsa_decode(num_requests=3, num_layers=3, steps=5, context=5000)
+    pair = Pair(w)
+    tr = inputs.Trace(w)
+    side = torch.cuda.Stream()
+    try:
+        for step in range(w.steps):
+            sel, app, _ = tr.step()
+            if app:
+                pair.append()
+            for layer in range(w.num_layers):
+                pair.resolve_and_compare(layer, sel[layer])
+                if layer + 1 < w.num_layers:
+                    hint = torch.from_numpy(np.ascontiguousarray(sel[layer])).to(pair.dev)
+                    pair.gpu.prefetch_hint(layer + 1, hint, side)
+                    pair.oracle.resolve(layer + 1, sel[layer])
+                pair.compare_state(layer)
+        pair.finish()
+    finally:
+        tr.close()
+        pair.close()
+    grouped = Pair(tiny_workload(3, 2, 2, 6, 10, 48, [40, 50, 60]))
+    try:
+        with pytest.raises(HiSparseError) as e:      # shared-selection groups use the exact prefetch instead
+            grouped.gpu.prefetch_hint(0, torch.zeros((3, 6), dtype=torch.int32, device="cuda"), side)
+        assert e.value.code == hs.EINVAL
+    finally:
+        grouped.close()
+
+
 # ------------------------------------------------------------------ CUDA graph replay of whole steps
 
 def test_graph_replay_matches_oracle():
