@@ -181,6 +181,46 @@ def oracle_throughput(w_full, n_req: int, steps: int, warmup: int):
     return sels / t_total, t_total / max(1, steps), per_step
 
 
+def oracle_throughput_parallel(w_full, n_req: int, steps: int, threads: int):
+    """The same oracle, one instance per request (requests are independent), spread over `threads` host threads
+    (ctypes releases the GIL inside the C calls).  Returns selections/s over the timed steps."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import Oracle
+    from paper_2608_07009_b200 import inputs
+    import copy
+    w = copy.copy(w_full)
+    w.num_requests = n_req
+    w.init_len = list(w_full.init_len[:n_req])
+    w.steps = 3 + steps
+    hist = [inputs.new_history(w, r) for r in range(n_req)]
+    orcs = [Oracle(1, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k, w.entry_bytes, [w.capacity[r]],
+                   [w.init_len[r]], [hist[r]]) for r in range(n_req)]
+    tr = inputs.Trace(w)
+    rows = [tr.step() for _ in range(2 + steps)]
+    tr.close()
+    kvs = [inputs.new_kv(w, lens - 1) if app else None for _, app, lens in rows]
+
+    def work(r, lo, hi):
+        n = 0
+        for s in range(lo, hi):
+            sel, app, _ = rows[s]
+            if app:
+                orcs[r].append(kvs[s][r:r + 1])
+            for layer in range(w.num_layers):
+                _, h, m = orcs[r].resolve(layer, sel[layer // w.layers_per_group][r:r + 1])
+                n += int(h[0]) + int(m[0])
+        return n
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        list(pool.map(lambda r: work(r, 0, 2), range(n_req)))            # cold step + one warm-up step
+        t0 = time.perf_counter()
+        done = sum(pool.map(lambda r: work(r, 2, 2 + steps), range(n_req)))
+        dt = time.perf_counter() - t0
+    for o in orcs:
+        o.close()
+    return done / dt
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -494,6 +534,13 @@ def run_ours(args):
             "value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": "requests 0..%d of %d, all %d layers, %d steps after the cold step and 1 warm-up step" % (
                 n_req - 1, N, L, steps_cpu)}
+        threads = min(os.cpu_count() or 1, N)
+        n_par = min(N, threads)
+        extra["cpu_baseline_parallel"] = {
+            "value": oracle_throughput_parallel(w, n_par, max(1, steps_cpu // 4), threads), "unit": UNIT,
+            "cores": threads, "kind": "oracle, one instance per request on a thread pool",
+            "sample": "requests 0..%d of %d, all %d layers, %d steps after the cold step and 1 warm-up step" % (
+                n_par - 1, N, L, max(1, steps_cpu // 4))}
     if launched:
         dist.barrier()
         dist.destroy_process_group()

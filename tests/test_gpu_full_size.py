@@ -5,20 +5,22 @@ The oracle tracks metadata only here (no second copy of tens of GB of history): 
 are compared for every request and layer, the full LRU state for sampled (request, layer) pairs, and the bytes by
 property — every table entry must address bytes equal to the host history (device-side compare of ALL selections)
 and, for sampled entries, equal to the generator's record computed one by one.
-C4 / C5 run with 4 of their 16 / 32 layers unless HISPARSE_FULL_LAYERS=1 (34 GB / 69 GB of pinned history
-otherwise); every other dimension is the configuration's own.
+C4 / C5 need 34 GB / 69 GB of pinned history at their full 16 / 32 layers.  They run at full size; if the host
+cannot pin that much (or HISPARSE_REDUCED_LAYERS=1 is set) they fall back, with a warning, to 4 layers, every
+other dimension being the configuration's own.
 """
 import os
+import warnings
 
 import numpy as np
 import pytest
 import torch
 
 from oracle import Oracle, FLAG_NO_BYTES
-from paper_2608_07009_b200 import HiSparse, HostHistory, inputs
+from paper_2608_07009_b200 import HiSparse, HostHistory, HiSparseError, inputs, hisparse as hs
 
 pytestmark = pytest.mark.gpu
-FULL_LAYERS = os.environ.get("HISPARSE_FULL_LAYERS", "0") == "1"
+REDUCED = os.environ.get("HISPARSE_REDUCED_LAYERS", "0") == "1"
 
 
 def run_full(w, steps, sample_pairs, use_prefetch=False):
@@ -26,7 +28,14 @@ def run_full(w, steps, sample_pairs, use_prefetch=False):
     N, L, lpg, G, k, B, E = (w.num_requests, w.num_layers, w.layers_per_group, w.num_groups, w.top_k,
                              w.cache_slots, w.entry_bytes)
     cap = w.capacity
-    hist = [HostHistory(L, cap[r], E) for r in range(N)]
+    hist = []
+    try:
+        for r in range(N):
+            hist.append(HostHistory(L, cap[r], E))
+    except HiSparseError:
+        for h in hist:
+            h.free()
+        raise
     for r, h in enumerate(hist):
         inputs.fill_history(h.ptr, r, L, cap[r], 0, w.init_len[r], E, w.seed)
     gpu = HiSparse(N, L, lpg, B, k, E, cap, w.init_len, hist)
@@ -117,11 +126,22 @@ def test_c3_dsa_long_full_size_with_prefetch():
     run_full(w, 3, [(0, 0), (8, 1), (8, 4), (3, 7)], use_prefetch=True)
 
 
+def full_or_reduced(make, steps, full_layers):
+    if not REDUCED:
+        try:
+            w = make(full_layers)
+            return run_full(w, steps, [(0, 0), (15, w.num_layers - 1)])
+        except HiSparseError as e:
+            if e.code != hs.ENOMEM:
+                raise
+            warnings.warn("could not pin %d layers of history: running the 4-layer variant" % full_layers)
+    w = make(4)
+    run_full(w, steps, [(0, 0), (15, w.num_layers - 1)])
+
+
 def test_c4_nsa_blocks_full_size():
-    w = inputs.c4_nsa_blocks(steps=66, num_layers=16 if FULL_LAYERS else 4)
-    run_full(w, 66, [(0, 0), (15, w.num_layers - 1)])
+    full_or_reduced(lambda layers: inputs.c4_nsa_blocks(steps=66, num_layers=layers), 66, 16)
 
 
 def test_c5_quest_pages_full_size():
-    w = inputs.c5_quest_pages(steps=17, num_layers=32 if FULL_LAYERS else 4)
-    run_full(w, 17, [(0, 0), (15, w.num_layers - 1)])
+    full_or_reduced(lambda layers: inputs.c5_quest_pages(steps=17, num_layers=layers), 17, 32)
