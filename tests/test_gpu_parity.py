@@ -343,3 +343,19 @@ def test_create_rejects_bad_arguments():
         assert kv == 1 * 1 * 9 * 32 and meta > 0
     finally:
         hist.free()
+
+
+# ------------------------------------------------------------------ the boundary from plain C
+
+def test_c_program_uses_the_library(tmp_path):
+    import os
+    import subprocess
+    from paper_2608_07009_b200 import build
+    root = build.ROOT
+    exe = str(tmp_path / "c_abi_smoke")
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    subprocess.check_call(["gcc", "-std=c99", os.path.join(root, "tests", "c_abi_smoke.c"), "-I", os.path.join(root, "include"),
+                           "-I", os.path.join(cuda, "include"), "-o", exe, build.SO, "-L", os.path.join(cuda, "lib64"),
+                           "-lcudart", "-Wl,-rpath," + os.path.dirname(build.SO), "-Wl,-rpath," + os.path.join(cuda, "lib64")])
+    out = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+    assert out.returncode == 0 and "C-ABI OK" in out.stdout, out.stdout + out.stderr
