@@ -49,6 +49,7 @@ constexpr int kFetchUnroll = 4;      // 16-byte host loads in flight per thread 
 constexpr int kBarBytes = (kThreads + 2) * 8;  // one mbarrier per thread for the fetch ring + one for staging
 constexpr int32_t kMiss = -2;        // s_out marker: valid selection, not (yet) found resident
 constexpr int32_t kDupBase = -3;     // s_out marker: duplicate of row entry -(v + 3)
+constexpr int32_t kRankBase = -(1 << 20);  // s_out marker: the (kRankBase - v)-th miss of the row (slot = plan_slot of it)
 
 // Everything a kernel needs, passed by value.
 struct DevState {
@@ -240,7 +241,8 @@ __device__ __forceinline__ void fetch_barriers_init(unsigned long long *bars, in
 
 // ------------------------------------------------------------------------------------------ Resolve (Sec. 3.4)
 
-// Block-wide exclusive prefix sum of one int per thread (two barriers).  s_warp: 32 ints of scratch.
+// Block-wide exclusive prefix sum of one int per thread (one barrier).  s_warp: 32 ints of scratch, which the
+// caller must not reuse (another scan included) before the block has passed a barrier of its own.
 __device__ __forceinline__ int block_scan_excl(int v, int *s_warp, int &total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
   int incl = v;
@@ -260,7 +262,6 @@ __device__ __forceinline__ int block_scan_excl(int v, int *s_warp, int &total) {
   }
   const int warp_excl = __shfl_sync(0xffffffffu, wincl - w, warp);
   total = __shfl_sync(0xffffffffu, wincl, 31);
-  __syncthreads();
   return warp_excl + incl - v;
 }
 
@@ -397,10 +398,10 @@ __device__ __forceinline__ void select_random_victims(const int B, const int m, 
 }
 
 // Everything the first block of a cluster does before the fetch can start: Phases 1-3 of Sec. 3.4.
-// IPT = entries of the recency order per thread (B <= IPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
+// IPT = entries of the recency order per thread (B <= IPT * kThreads), KPT = row entries per thread (k <= KPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
 // the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
 // the untouched slots compacted at its front, and s_hitbits / s_vicbits the per-slot marks.
-template <int IPT>
+template <int IPT, int KPT>
 __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r, const int64_t rg, const int32_t *row,
                                                  int32_t *s_sel, int32_t *s_out, int32_t *s_plan_pos,
                                                  int32_t *s_plan_slot, unsigned long long *s_tab, uint32_t *s_hitbits,
@@ -415,26 +416,45 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   const int k = d.k, B = d.B, H = d.H;
   const uint32_t mask = (uint32_t)(H - 1);
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+  bool timed_out = false;
 
   // Phase 1: stage the row and the recency order (one round trip to HBM).  The request's slice of the page
   // table is streamed into the (still idle) fetch ring with bulk copies when it fits, so that Phase 2's k random
   // lookups hit shared memory instead of queueing as 32-byte sector reads on one SM.
-  stage_async(s_sel, row, k * 4);
-  stage_async(s_order, d.order + rg * B, B * 2);
   const int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)(rg - (int64_t)r * d.G) * cap_r;
   const uintptr_t p2s_aligned = (uintptr_t)p2s & ~(uintptr_t)15;
   const int lead = (int)(((uintptr_t)p2s - p2s_aligned) >> 1);
   const int64_t stage_bytes = ((int64_t)lead * 2 + cap_r * 2) & ~(int64_t)15;  // whole 16-byte units only
   const bool staged = stage_bytes + 16 <= (int64_t)d.ring_bytes;
   const uint32_t stage_bar = smem_u32(s_bars + kThreads);
-  if (staged && tid == 0) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(stage_bar), "r"((uint32_t)stage_bytes) : "memory");
-    for (int64_t o = 0; o < stage_bytes; o += 32768) {
-      const uint32_t n = (uint32_t)(stage_bytes - o < 32768 ? stage_bytes - o : 32768);
+  const uint16_t *order_g = d.order + rg * B;
+  // 16-byte aligned arrays are fetched by ONE thread with bulk copies (a handful of instructions for the whole
+  // block); anything else falls back to per-thread cp.async
+  const bool sel_bulk = (((uintptr_t)row | (uintptr_t)(k * 4)) & 15) == 0;
+  const bool ord_bulk = (((uintptr_t)order_g | (uintptr_t)(B * 2)) & 15) == 0;
+  // one expect_tx for everything; each copy is issued by the first lane of a different warp, so that the copies
+  // enter the bulk-copy engine side by side (a copy that lands before the expect_tx only makes the count dip)
+  if (tid == 0) {
+    const uint32_t tx = (sel_bulk ? (uint32_t)k * 4u : 0u) + (ord_bulk ? (uint32_t)B * 2u : 0u) +
+                        (staged ? (uint32_t)stage_bytes : 0u);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(stage_bar), "r"(tx) : "memory");
+    if (sel_bulk)
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(s_sel)), "l"(row), "r"((uint32_t)k * 4u), "r"(stage_bar) : "memory");
+  }
+  if (tid == 32 && ord_bulk)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(s_order)), "l"(order_g), "r"((uint32_t)B * 2u), "r"(stage_bar) : "memory");
+  if (staged && tid >= 64 && (tid & 31) == 0) {
+    constexpr int kPiece = 16384;
+    for (int64_t o = (int64_t)((tid >> 5) - 2) * kPiece; o < stage_bytes; o += (int64_t)(kThreads / 32 - 2) * kPiece) {
+      const uint32_t n = (uint32_t)(stage_bytes - o < kPiece ? stage_bytes - o : kPiece);
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                    ::"r"(smem_u32(s_ring) + (uint32_t)o), "l"((const char *)p2s_aligned + o), "r"(n), "r"(stage_bar) : "memory");
     }
   }
+  if (!sel_bulk) stage_async(s_sel, row, k * 4);
+  if (!ord_bulk) stage_async(s_order, order_g, B * 2);
   if (staged && tid >= 32 && tid < 40) {  // the last, partial 16-byte unit of the slice: plain copies
     const int64_t e = stage_bytes / 2 + (tid - 32);
     if (e < lead + cap_r) reinterpret_cast<int16_t *>(s_ring)[e] = reinterpret_cast<const int16_t *>(p2s_aligned)[e];
@@ -443,11 +463,13 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
   const int64_t newest = (na > 0 && init_len_r + na <= cap_r) ? init_len_r + na - 1 : -1;
   if (timers && tid == 0) stamps[8] = clock64();
-  asm volatile("cp.async.wait_all;" ::: "memory");
+  if (!sel_bulk || !ord_bulk) asm volatile("cp.async.wait_all;" ::: "memory");
   bool use_staged = staged;
-  if (staged && !mbar_wait_bounded(stage_bar, 0u)) {
-    use_staged = false;  // bounded wait expired: fall back to the table in HBM
+  if (!mbar_wait_bounded(stage_bar, 0u)) {
+    // bounded wait expired: the row cannot be trusted either, so this request resolves nothing in this launch
+    use_staged = false;
     my_status |= HISPARSE_STATUS_TIMEOUT;
+    timed_out = true;
   }
   __syncthreads();
   if (timers && tid == 0) stamps[9] = clock64();
@@ -457,11 +479,11 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
   // resident go into the hash table (position -> row index), whose only job is to catch a position that is
   // selected twice, so that it claims one victim, not two.
-  int32_t pos[kSelPerThread], got[kSelPerThread];
+  int32_t pos[KPT], got[KPT];
 #pragma unroll
-  for (int i = 0; i < kSelPerThread; ++i) {
+  for (int i = 0; i < KPT; ++i) {
     const int j = tid + i * T;
-    pos[i] = j < k ? s_sel[j] : -1;
+    pos[i] = (j < k && !timed_out) ? s_sel[j] : -1;
     const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
     if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
     if (!ok) pos[i] = -1;
@@ -469,7 +491,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
 #pragma unroll
-  for (int i = 0; i < kSelPerThread; ++i) {
+  for (int i = 0; i < KPT; ++i) {
     const int j = tid + i * T;
     if (j >= k) break;
     const int32_t p = pos[i];
@@ -517,13 +539,12 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
         }
       }
     }
+    __syncthreads();
   }
-  if (timers && tid == 0) stamps[11] = clock64();
-  __syncthreads();
-  if (timers && tid == 0) stamps[12] = clock64();
+  if (timers && tid == 0) { stamps[11] = clock64(); stamps[12] = stamps[11]; }
 
   // Phase 3: ONE block scan over packed counts (non-hit slots in recency order | misses in selection order).
-  // Thread t owns IPT consecutive entries of the recency order and kSelPerThread consecutive row entries.
+  // Thread t owns IPT consecutive entries of the recency order and KPT consecutive row entries.
   {
     int slot[IPT];
     uint32_t nh_mask = 0, miss_mask = 0;
@@ -537,8 +558,8 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
       }
     }
 #pragma unroll
-    for (int i = 0; i < kSelPerThread; ++i) {
-      const int j = tid * kSelPerThread + i;
+    for (int i = 0; i < KPT; ++i) {
+      const int j = tid * KPT + i;
       if (j < k && s_out[j] == kMiss) miss_mask |= 1u << i;
     }
     int total;
@@ -547,8 +568,13 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     n_nonhit = total >> 16;
     int mrank = excl & 0xffff, nrank = excl >> 16;
 #pragma unroll
-    for (int i = 0; i < kSelPerThread; ++i)
-      if ((miss_mask >> i) & 1u) s_plan_pos[mrank++] = tid * kSelPerThread + i;
+    for (int i = 0; i < KPT; ++i)
+      if ((miss_mask >> i) & 1u) {
+        const int j = tid * KPT + i;
+        s_plan_pos[mrank] = s_sel[j];      // position of the mrank-th miss
+        s_out[j] = kRankBase - mrank;      // its slot is the mrank-th victim, looked up when the table is written
+        ++mrank;
+      }
     if (d.policy == HISPARSE_POLICY_LRU) {
       // the i-th miss (selection order) takes the i-th non-hit slot of the recency order
 #pragma unroll
@@ -619,12 +645,6 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   }
   if (timers && tid == 0) stamps[13] = clock64();
   __syncthreads();
-  for (int i = tid; i < m; i += T) {
-    const int j = s_plan_pos[i];
-    s_out[j] = s_plan_slot[i];
-    s_plan_pos[i] = s_sel[j];
-  }
-  __syncthreads();
   if (timers && tid == 0) stamps[14] = clock64();
 }
 
@@ -675,12 +695,19 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     const uint32_t miss_stamp = 2u * t;
     uint32_t my_status = 0;
     const int32_t *row = sel + (int64_t)r * k;
-#define HS_META(IPT)                                                                                              \
-  resolve_metadata<IPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits, s_order, \
-                        s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t, s_vicpre, m, n_nonhit, my_status)
-    if (B <= 4 * T) HS_META(4);
-    else if (B <= 8 * T) HS_META(8);
-    else HS_META(16);
+#define HS_META(IPT, KPT)                                                                                         \
+  resolve_metadata<IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
+                             s_order, s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t,      \
+                             s_vicpre, m, n_nonhit, my_status)
+    if (k <= 2 * T) {
+      if (B <= 4 * T) HS_META(4, 2);
+      else if (B <= 8 * T) HS_META(8, 2);
+      else HS_META(16, 2);
+    } else {
+      if (B <= 4 * T) HS_META(4, kSelPerThread);
+      else if (B <= 8 * T) HS_META(8, kSelPerThread);
+      else HS_META(16, kSelPerThread);
+    }
 #undef HS_META
     if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
     // Phase 4 starts here: the first batch of host loads is in flight while the metadata is written back
@@ -736,7 +763,8 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     int32_t *arow = d.anchor_out + rg * k;
     for (int j = tid; j < k; j += T) {
       int32_t o = s_out[j];
-      if (o <= kDupBase) o = s_out[kDupBase - o];
+      if (o <= kDupBase && o > kRankBase) o = s_out[kDupBase - o];  // a repeated position follows its first occurrence
+      if (o <= kRankBase) o = s_plan_slot[kRankBase - o];           // a miss takes its victim's slot
       trow[j] = o < 0 ? -1 : r * (B + 1) + o;
       if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
     }
