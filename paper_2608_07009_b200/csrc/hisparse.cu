@@ -685,6 +685,20 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     if (tid < 4) s_misc[tid] = 0;
   }
   const int64_t cap_r = d.cap[r], init_len_r = d.init_len[r], p2s_off_r = d.p2s_off[r];  // fixed at create
+  if (part == 0 && tid < 3) {
+    // Warm L2 with what Phase 1 will stage (row, recency order, page-table slice).  A prefetch consumes nothing, and
+    // L2 is where earlier kernels' writes land, so this is safe before the dependency wait; when the previous kernel
+    // lets its dependents start early, the staging after the wait then reads L2 instead of HBM.
+    const char *p = tid == 0 ? reinterpret_cast<const char *>(sel + (int64_t)r * k)
+                  : tid == 1 ? reinterpret_cast<const char *>(d.order + rg * B)
+                             : reinterpret_cast<const char *>(d.pos2slot + p2s_off_r + (int64_t)g * cap_r);
+    int64_t n = tid == 0 ? (int64_t)k * 4 : tid == 1 ? (int64_t)B * 2 : cap_r * 2;
+    const uintptr_t a = ((uintptr_t)p + 15) & ~(uintptr_t)15;   // whole 16-byte units inside the array only
+    n = (n - (int64_t)(a - (uintptr_t)p)) & ~(int64_t)15;
+    if (n > (1 << 20)) n = 1 << 20;                             // no point warming more than the ring could stage
+    if (n > 0)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a), "r"((uint32_t)n) : "memory");
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   TmaFetch fetch;
   int m = 0, n_nonhit = 0;
