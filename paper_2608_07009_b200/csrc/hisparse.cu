@@ -397,6 +397,47 @@ __device__ __forceinline__ void select_random_victims(const int B, const int m, 
   __syncthreads();
 }
 
+
+// Page-table lookups shared by the blocks of a cluster (used when a request's slice of the table is too large to
+// stage in shared memory: k uncoalesced reads are bound by one SM's load path, so each block of the cluster does
+// k/S of them).  Block `part` answers row entries [part*chunk, (part+1)*chunk) and stores the answers (slot, or -1
+// for padding / out of range / host-only) into the FIRST block's s_got through distributed shared memory.
+// Cluster barrier phases: every block arrives on phase A when it starts; a block stores into the first block's
+// memory only after waiting for phase A (all blocks are running by then); phase B = all answers are in.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// phase A only says "this block is running": no memory needs to be ordered by it
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_relaxed() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void cluster_lookups(const int32_t *__restrict__ row, const int16_t *__restrict__ p2s,
+                                                const int k, const int64_t len, const int part, const int S,
+                                                int16_t *s_got) {
+  constexpr int kMaxPer = (HISPARSE_MAX_TOP_K / 2 + kThreads - 1) / kThreads;  // S >= 2, so a block's share <= k/2
+  const int chunk = (k + S - 1) / S;
+  const int lo = part * chunk, hi = lo + chunk < k ? lo + chunk : k;
+  int16_t v[kMaxPer];
+#pragma unroll
+  for (int i = 0; i < kMaxPer; ++i) {
+    const int j = lo + (int)threadIdx.x + i * kThreads;
+    v[i] = -1;
+    if (j < hi) {
+      const int32_t p = __ldg(row + j);
+      if (p >= 0 && (int64_t)p < len) v[i] = __ldg(p2s + p);
+    }
+  }
+  cluster_wait_relaxed();  // phase A: the first block is running, its shared memory may be written
+  uint32_t remote_base;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote_base) : "r"(smem_u32(s_got)), "r"(0));
+#pragma unroll
+  for (int i = 0; i < kMaxPer; ++i) {
+    const int j = lo + (int)threadIdx.x + i * kThreads;
+    if (j < hi) asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(remote_base + 2u * (uint32_t)j), "h"(v[i]) : "memory");
+  }
+  cluster_arrive();  // phase B
+  cluster_wait();
+}
+
 // Everything the first block of a cluster does before the fetch can start: Phases 1-3 of Sec. 3.4.
 // IPT = entries of the recency order per thread (B <= IPT * kThreads), KPT = row entries per thread (k <= KPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
 // the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
@@ -409,8 +450,8 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  const int64_t cap_r, const int64_t init_len_r,
                                                  const int64_t p2s_off_r, unsigned long long *stamps,
                                                  unsigned char *s_ring, unsigned long long *s_bars,
-                                                 const uint32_t t_now, int *s_warp_pre, int &m, int &n_nonhit,
-                                                 uint32_t &my_status) {
+                                                 const uint32_t t_now, int *s_warp_pre, int16_t *s_got, const int S,
+                                                 int &m, int &n_nonhit, uint32_t &my_status) {
   constexpr int T = kThreads;
   const int tid = threadIdx.x;
   const int k = d.k, B = d.B, H = d.H;
@@ -426,6 +467,8 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   const int lead = (int)(((uintptr_t)p2s - p2s_aligned) >> 1);
   const int64_t stage_bytes = ((int64_t)lead * 2 + cap_r * 2) & ~(int64_t)15;  // whole 16-byte units only
   const bool staged = stage_bytes + 16 <= (int64_t)d.ring_bytes;
+  const bool coop = !staged && S > 1;  // same decision in every block of the cluster (depends on the request only)
+  if (coop) cluster_arrive_relaxed();  // phase A, see cluster_lookups
   const uint32_t stage_bar = smem_u32(s_bars + kThreads);
   const uint16_t *order_g = d.order + rg * B;
   // 16-byte aligned arrays are fetched by ONE thread with bulk copies (a handful of instructions for the whole
@@ -474,6 +517,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   __syncthreads();
   if (timers && tid == 0) stamps[9] = clock64();
   const int16_t *s_p2s = reinterpret_cast<const int16_t *>(s_ring) + lead;
+  if (coop) cluster_lookups(row, p2s, k, len, 0, S, s_got);
 
   // Phase 2: hit detection through the page table (position -> slot): all of a thread's lookups are issued
   // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
@@ -487,7 +531,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
     if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
     if (!ok) pos[i] = -1;
-    got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : __ldg(p2s + pos[i]));
+    got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : coop ? s_got[j] : __ldg(p2s + pos[i]));
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
 #pragma unroll
@@ -673,6 +717,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   int32_t *s_hitpre = reinterpret_cast<int32_t *>(s_vicbits + W);
   int32_t *s_vicpre = s_hitpre + W;
   uint16_t *s_order = reinterpret_cast<uint16_t *>(s_vicpre + W);
+  int16_t *s_got = reinterpret_cast<int16_t *>(s_order + ((B + 7) & ~7));  // page-table answers from the whole cluster
   unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
   unsigned char *s_ring = smem_raw + d.meta_smem + kBarBytes;
 
@@ -703,6 +748,18 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   TmaFetch fetch;
   int m = 0, n_nonhit = 0;
   uint32_t t = 0;
+  if (part != 0) {
+    // same test as in resolve_metadata: is this request's page-table slice too large to be staged?
+    const int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
+    const int lead = (int)((((uintptr_t)p2s) & 15) >> 1);
+    const int64_t stage_bytes = ((int64_t)lead * 2 + cap_r * 2) & ~(int64_t)15;
+    if (!(stage_bytes + 16 <= (int64_t)d.ring_bytes)) {
+      const int64_t na = *(volatile int32_t *)d.n_appends;
+      const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
+      cluster_arrive_relaxed();  // phase A
+      cluster_lookups(sel + (int64_t)r * k, p2s, k, len, part, S, s_got);
+    }
+  }
   if (part == 0) {
     if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
     t = d.t[rg] + 1u;
@@ -712,7 +769,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
 #define HS_META(IPT, KPT)                                                                                         \
   resolve_metadata<IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
                              s_order, s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t,      \
-                             s_vicpre, m, n_nonhit, my_status)
+                             s_vicpre, s_got, S, m, n_nonhit, my_status)
     if (k <= 2 * T) {
       if (B <= 4 * T) HS_META(4, 2);
       else if (B <= 8 * T) HS_META(8, 2);
@@ -1109,7 +1166,7 @@ int hash_size(int k) {
 
 size_t resolve_smem_bytes(int B, int k) {
   const int H = hash_size(k), W = (B + 31) / 32;
-  return (size_t)H * 8 + (size_t)4 * k * 4 + (size_t)4 * W * 4 + (size_t)B * 2;
+  return (size_t)H * 8 + (size_t)4 * k * 4 + (size_t)4 * W * 4 + (size_t)((B + 7) & ~7) * 2 + (size_t)k * 2;
 }
 
 cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }

@@ -163,6 +163,14 @@ def test_c3_shape_reduced_with_prefetch(overlap):
     run_trace(w, w.steps, use_prefetch=True, flags=hs.FLAG_DEBUG_VALIDATE)
 
 
+@pytest.mark.parametrize("S", [1, 2, 8])
+def test_long_context_page_table_not_staged(S):
+    # page-table slices of 180 KB and 400 KB do not fit the staging ring: the blocks of a cluster share the lookups
+    w = inputs.c3_dsa_long(0.5, steps=4, short_ctx=90000, long_ctx=200000, num_short=2)
+    w.entry_bytes = 64
+    run_trace(w, w.steps, use_prefetch=True, ctas_per_request=S, flags=hs.FLAG_DEBUG_VALIDATE)
+
+
 def test_c4_nsa_blocks_reduced():
     w = inputs.c4_nsa_blocks(num_requests=4, num_layers=2, steps=70)
     w.entry_bytes = 16384            # same block-granular selection, smaller blocks
