@@ -208,6 +208,13 @@ int hisparse_device_bytes(const hisparse_config_t *cfg, size_t *kv_bytes, size_t
  * classified, [11] / [12] counted, before / after the barrier, [13] scanned, [14] plan ready.  Synchronises. */
 int hisparse_phase_times(hisparse_t *h, uint64_t *out);
 
+/* Failure-detection self-test.  Every device-side wait of the library (on the mbarriers of its bulk copies) is
+ * bounded: after 2 s it gives up, sets STATUS_TIMEOUT and the kernel returns, so a lost completion can never hang
+ * the GPU.  This call runs that very wait on a barrier that nothing completes, with a limit of limit_ns
+ * (<= 1 s): it must return after about that long with STATUS_TIMEOUT set (clear it with hisparse_clear_status)
+ * and the handle still usable.  *waited_ns receives the time the kernel spent waiting.  Synchronises. */
+int hisparse_selftest_wait_timeout(hisparse_t *h, uint64_t limit_ns, uint64_t *waited_ns);
+
 /* Launch geometry chosen at create: thread blocks per request and threads per block. */
 int hisparse_launch_geometry(const hisparse_t *h, int32_t *ctas_per_request, int32_t *threads, int32_t *smem_bytes);
 

@@ -120,7 +120,8 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                  unsigned long long limit_ns = 2000000000ull) {
   uint32_t done = 0;
   uint64_t t0 = 0;
   for (uint32_t spin = 0;; ++spin) {
@@ -130,7 +131,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     if ((spin & 63u) == 63u) {
       const uint64_t now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > 2000000000ull) return false;
+      else if (now - t0 > limit_ns) return false;
     }
   }
 }
@@ -1068,6 +1069,20 @@ __global__ void validate_kernel(const DevState d, const int g) {
   if (bad) atomicOr(d.status, HISPARSE_STATUS_INCONSISTENT);
 }
 
+// Exercises the bounded wait on purpose: an mbarrier that nothing ever completes.  The wait gives up after
+// limit_ns, sets STATUS_TIMEOUT and the kernel returns normally; *waited_ns receives how long it waited.
+__global__ void wait_timeout_selftest_kernel(uint32_t *status, unsigned long long limit_ns,
+                                             unsigned long long *waited_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const unsigned long long t0 = global_ns();
+    if (!mbar_wait_bounded(smem_u32(&bar), 0u, limit_ns)) atomicOr(status, HISPARSE_STATUS_TIMEOUT);
+    *waited_ns = global_ns() - t0;
+  }
+}
+
 __global__ void init_order_kernel(uint16_t *order, int64_t n, int B) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     order[i] = (uint16_t)(i % B);
@@ -1606,6 +1621,16 @@ int hisparse_phase_times(hisparse_t *h, uint64_t *out) {
   HS_CUDA(cudaSetDevice(h->device));
   HS_CUDA(cudaDeviceSynchronize());
   HS_CUDA(cudaMemcpy(out, h->d.phase_ns, (size_t)h->d.N * 16 * 8, cudaMemcpyDeviceToHost));
+  return HISPARSE_OK;
+}
+
+int hisparse_selftest_wait_timeout(hisparse_t *h, uint64_t limit_ns, uint64_t *waited_ns) {
+  if (!h || !waited_ns || limit_ns == 0 || limit_ns > 1000000000ull) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  wait_timeout_selftest_kernel<<<1, 32>>>(h->d.status, limit_ns, h->d.phase_ns);
+  HS_CUDA(cudaGetLastError());
+  HS_CUDA(cudaDeviceSynchronize());
+  HS_CUDA(cudaMemcpy(waited_ns, h->d.phase_ns, 8, cudaMemcpyDeviceToHost));
   return HISPARSE_OK;
 }
 

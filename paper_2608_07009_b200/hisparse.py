@@ -25,7 +25,7 @@ EXPORTS = [
     "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch", "hisparse_prefetch_hint",
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
     "hisparse_clear_status", "hisparse_dump_state", "hisparse_dump_plan", "hisparse_device_bytes",
-    "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
+    "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_selftest_wait_timeout", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
     "hisparse_scatter_read_probe", "hisparse_resolve_noalloc", "hisparse_strerror", "hisparse_last_cuda_error",
 ]
 
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
             "hisparse_device_bytes": ([P(Config), P(sz), P(sz)], i32),
             "hisparse_launch_geometry": ([vp, P(ctypes.c_int32), P(ctypes.c_int32), P(ctypes.c_int32)], i32),
             "hisparse_phase_times": ([vp, vp], i32),
+            "hisparse_selftest_wait_timeout": ([vp, ctypes.c_uint64, P(ctypes.c_uint64)], i32),
             "hisparse_host_alloc": ([sz, P(vp)], i32),
             "hisparse_host_free": ([vp], i32),
             "hisparse_host_link_probe": ([i32, sz, i32, P(ctypes.c_double)], i32),
@@ -312,6 +313,12 @@ class HiSparse:
         out = np.zeros((self.N, 16), dtype=np.uint64)
         _check(lib().hisparse_phase_times(self._h, out.ctypes.data), "hisparse_phase_times")
         return out
+
+    def selftest_wait_timeout(self, limit_ns: int) -> int:
+        """Runs the library's bounded wait on a barrier that never completes; returns the nanoseconds waited."""
+        out = ctypes.c_uint64()
+        _check(lib().hisparse_selftest_wait_timeout(self._h, limit_ns, ctypes.byref(out)), "hisparse_selftest_wait_timeout")
+        return out.value
 
     def launch_geometry(self):
         s, t, m = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()

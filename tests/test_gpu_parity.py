@@ -320,6 +320,24 @@ def test_graph_replay_matches_oracle():
         pair.close()
 
 
+# ------------------------------------------------------------------ failure detection without a fault
+
+def test_bounded_wait_expires_and_the_handle_stays_usable():
+    w = tiny_workload(2, 1, 1, 4, 8, 32, [20, 30])
+    pair = Pair(w)
+    try:
+        pair.resolve_and_compare(0, np.array([[1, 2, 3, 4], [5, 6, 7, 8]]))
+        waited = pair.gpu.selftest_wait_timeout(2_000_000)              # a barrier nothing completes, 2 ms limit
+        assert 2_000_000 <= waited < 200_000_000
+        assert pair.gpu.status() == hs.STATUS_TIMEOUT                    # reported, not hung, no fault
+        pair.gpu.clear_status()
+        pair.resolve_and_compare(0, np.array([[4, 9, 1, -1], [8, 7, 0, 29]]))   # the context is intact
+        pair.compare_state(0)
+        pair.finish()
+    finally:
+        pair.close()
+
+
 # ------------------------------------------------------------------ boundary errors
 
 def test_create_rejects_bad_arguments():
