@@ -192,6 +192,17 @@ int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, ui
                         int32_t *lru_order, int32_t *pos2slot, int64_t *len, int64_t *newest,
                         uint32_t *resolves);
 
+/* Checkpoint / resume, the counterparts of hisparse_dump_state (the paper has no such step; its scheduler only
+ * releases state).  hisparse_load_appends sets how many records every request has appended so far (lengths =
+ * init_len + appends; the histories must already hold those records).  hisparse_load_state then installs
+ * slot_pos [B] and last_use [B] (host arrays as dumped) as the metadata of (req, layer's group): it rebuilds the page
+ * table and the recency order from them, sets the resolve counter, and refills the cache of every layer of the
+ * group from the host history, which is authoritative (resident records and the newest record's reserved slot).
+ * EINVAL if a position is out of range or held by two slots.  Call between steps; synchronises. */
+int hisparse_load_appends(hisparse_t *h, int32_t appends);
+int hisparse_load_state(hisparse_t *h, int req, int layer, const int32_t *slot_pos, const uint32_t *last_use,
+                        uint32_t resolves);
+
 /* Miss plan recorded by the last resolve of `layer`'s anchor for request req: plan_pos / plan_slot
  * are host int32 [k]; *n receives the number of entries.  Synchronises. */
 int hisparse_dump_plan(hisparse_t *h, int req, int layer, int32_t *plan_pos, int32_t *plan_slot, int32_t *n);

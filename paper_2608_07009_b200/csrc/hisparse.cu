@@ -1605,6 +1605,63 @@ int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, ui
   return HISPARSE_OK;
 }
 
+int hisparse_load_state(hisparse_t *h, int req, int layer, const int32_t *slot_pos, const uint32_t *last_use,
+                        uint32_t resolves) {
+  if (!h || req < 0 || req >= h->d.N || layer < 0 || layer >= h->d.L || !slot_pos || !last_use) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  const int B = h->d.B, lpg = h->d.lpg, g = layer / lpg;
+  const int64_t rg = (int64_t)req * h->d.G + g, cap = h->cap[req];
+  int32_t na = 0;
+  HS_CUDA(cudaMemcpy(&na, h->d.n_appends, 4, cudaMemcpyDeviceToHost));
+  const int64_t len = std::min(h->init_len[req] + na, cap);
+  // the page table is the inverse of slot_pos; positions must be distinct and inside the history
+  std::vector<int16_t> p2s((size_t)cap, (int16_t)-1);
+  for (int s = 0; s < B; ++s) {
+    const int32_t p = slot_pos[s];
+    if (p == -1) continue;
+    if (p < 0 || p >= len || p2s[(size_t)p] != -1) return HISPARSE_EINVAL;
+    p2s[(size_t)p] = (int16_t)s;
+  }
+  // the recency order is the slots sorted by (stamp, slot)
+  std::vector<uint16_t> order((size_t)B);
+  for (int s = 0; s < B; ++s) order[(size_t)s] = (uint16_t)s;
+  std::stable_sort(order.begin(), order.end(), [&](uint16_t a, uint16_t b) { return last_use[a] < last_use[b]; });
+  HS_CUDA(cudaMemcpy(h->d.slot_pos + rg * B, slot_pos, (size_t)B * 4, cudaMemcpyHostToDevice));
+  HS_CUDA(cudaMemcpy(h->d.last_use + rg * B, last_use, (size_t)B * 4, cudaMemcpyHostToDevice));
+  HS_CUDA(cudaMemcpy(h->d.order + rg * B, order.data(), (size_t)B * 2, cudaMemcpyHostToDevice));
+  HS_CUDA(cudaMemcpy(h->d.pos2slot + h->p2s_off[req] + (int64_t)g * cap, p2s.data(), (size_t)cap * 2, cudaMemcpyHostToDevice));
+  HS_CUDA(cudaMemcpy(h->d.t + rg, &resolves, 4, cudaMemcpyHostToDevice));
+  const int32_t zero = 0;
+  HS_CUDA(cudaMemcpy(h->d.plan_n + rg, &zero, 4, cudaMemcpyHostToDevice));
+  // the host history is authoritative: refill every layer of the group from it (resident records + newest record)
+  cudaPointerAttributes a;
+  HS_CUDA(cudaPointerGetAttributes(&a, h->d.pool));
+  (void)a;
+  std::vector<uint8_t *> host(h->d.N);
+  HS_CUDA(cudaMemcpy(host.data(), h->d_host, sizeof(uint8_t *) * h->d.N, cudaMemcpyDeviceToHost));
+  const int64_t E = h->d.E;
+  for (int l = g * lpg; l < (g + 1) * lpg; ++l) {
+    uint8_t *pool = h->d.pool + (int64_t)l * h->d.layer_pool_bytes + (int64_t)req * (B + 1) * E;
+    const uint8_t *hist = host[req] + (int64_t)l * cap * E;   // device-visible alias of the pinned history
+    for (int s = 0; s < B; ++s)
+      if (slot_pos[s] >= 0)
+        HS_CUDA(cudaMemcpyAsync(pool + (int64_t)s * E, hist + (int64_t)slot_pos[s] * E, (size_t)E, cudaMemcpyDefault, nullptr));
+    if (na > 0 && h->init_len[req] + na <= cap)
+      HS_CUDA(cudaMemcpyAsync(pool + (int64_t)B * E, hist + (len - 1) * E, (size_t)E, cudaMemcpyDefault, nullptr));
+  }
+  HS_CUDA(cudaDeviceSynchronize());
+  return HISPARSE_OK;
+}
+
+int hisparse_load_appends(hisparse_t *h, int32_t appends) {
+  if (!h || appends < 0) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  HS_CUDA(cudaMemcpy(h->d.n_appends, &appends, 4, cudaMemcpyHostToDevice));
+  return HISPARSE_OK;
+}
+
 int hisparse_dump_plan(hisparse_t *h, int req, int layer, int32_t *plan_pos, int32_t *plan_slot, int32_t *n) {
   if (!h || req < 0 || req >= h->d.N || layer < 0 || layer >= h->d.L || !n) return HISPARSE_EINVAL;
   HS_CUDA(cudaSetDevice(h->device));

@@ -24,7 +24,7 @@ POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2
 EXPORTS = [
     "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch", "hisparse_prefetch_hint",
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
-    "hisparse_clear_status", "hisparse_dump_state", "hisparse_dump_plan", "hisparse_device_bytes",
+    "hisparse_clear_status", "hisparse_dump_state", "hisparse_load_state", "hisparse_load_appends", "hisparse_dump_plan", "hisparse_device_bytes",
     "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_selftest_wait_timeout", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
     "hisparse_scatter_read_probe", "hisparse_resolve_noalloc", "hisparse_strerror", "hisparse_last_cuda_error",
 ]
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
             "hisparse_status": ([vp, P(u32)], i32),
             "hisparse_clear_status": ([vp], i32),
             "hisparse_dump_state": ([vp, i32, i32, vp, vp, vp, vp, P(i64), P(i64), P(u32)], i32),
+            "hisparse_load_state": ([vp, i32, i32, vp, vp, u32], i32),
+            "hisparse_load_appends": ([vp, ctypes.c_int32], i32),
             "hisparse_dump_plan": ([vp, i32, i32, vp, vp, P(ctypes.c_int32)], i32),
             "hisparse_device_bytes": ([P(Config), P(sz), P(sz)], i32),
             "hisparse_launch_geometry": ([vp, P(ctypes.c_int32), P(ctypes.c_int32), P(ctypes.c_int32)], i32),
@@ -299,6 +301,16 @@ class HiSparse:
                "hisparse_dump_state")
         return dict(slot_pos=slot_pos, last_use=last_use, lru_order=order, pos2slot=p2s, len=ln.value,
                     newest=newest.value, resolves=t.value)
+
+    def load_appends(self, appends: int) -> None:
+        _check(lib().hisparse_load_appends(self._h, appends), "hisparse_load_appends")
+
+    def load_state(self, req: int, layer: int, slot_pos: np.ndarray, last_use: np.ndarray, resolves: int) -> None:
+        sp = np.ascontiguousarray(slot_pos, dtype=np.int32)
+        lu = np.ascontiguousarray(last_use, dtype=np.uint32)
+        assert sp.size == self.B and lu.size == self.B
+        _check(lib().hisparse_load_state(self._h, req, layer, sp.ctypes.data, lu.ctypes.data, resolves),
+               "hisparse_load_state")
 
     def dump_plan(self, req: int, layer: int):
         pos = np.empty(self.k, dtype=np.int32)

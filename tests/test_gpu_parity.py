@@ -320,6 +320,47 @@ def test_graph_replay_matches_oracle():
         pair.close()
 
 
+# ------------------------------------------------------------------ checkpoint / resume
+
+def test_dump_then_load_state_resumes_exactly():
+    w = inputs.c3_dsa_long(0.75, steps=8, short_ctx=3000, long_ctx=9000, num_short=2)     # 2 groups of 4 layers
+    w.entry_bytes = 64
+    pair = Pair(w)
+    tr = inputs.Trace(w)
+    N, L, lpg = w.num_requests, w.num_layers, w.layers_per_group
+    try:
+        for step in range(8):
+            sel, app, _ = tr.step()
+            if step == 4:
+                # checkpoint every (request, group), then bring up a fresh handle over the same host histories
+                pair.gpu.join()
+                snap = {(r, a): pair.gpu.dump_state(r, a) for r in range(N) for a in range(0, L, lpg)}
+                appends = snap[(0, 0)]["len"] - w.init_len[0]
+                old = pair.gpu
+                pair.gpu = HiSparse(N, L, lpg, w.cache_slots, w.top_k, w.entry_bytes, w.capacity, w.init_len,
+                                    pair.hist_gpu)
+                old.close()
+                pair.gpu.load_appends(appends)
+                for (r, a), st in snap.items():
+                    pair.gpu.load_state(r, a, st["slot_pos"], st["last_use"], st["resolves"])
+                for layer in range(L):
+                    pair.compare_whole_pool(layer)
+            if app:
+                pair.append()
+            for layer in range(L):
+                pair.resolve_and_compare(layer, sel[layer // lpg])
+                pair.compare_state(layer)
+        pair.finish()
+        bad = snap[(0, 0)]["slot_pos"].copy()
+        bad[1] = bad[0]
+        with pytest.raises(HiSparseError) as e:
+            pair.gpu.load_state(0, 0, bad, snap[(0, 0)]["last_use"], 1)
+        assert e.value.code == hs.EINVAL
+    finally:
+        tr.close()
+        pair.close()
+
+
 # ------------------------------------------------------------------ failure detection without a fault
 
 def test_bounded_wait_expires_and_the_handle_stays_usable():
