@@ -1,0 +1,57 @@
+"""Randomised parity soak: seeded random geometries (B, k, N, layer groups, record sizes, context lengths on both
+sides of the page-table staging limit), cluster sizes, replacement policies, padding and repeated positions — every
+step compared bit for bit with the oracle (tables, counts, LRU state, plans, bytes)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_07009_b200 import inputs, hisparse as hs
+from gpu_harness import Pair
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_random_configurations(seed):
+    rng = np.random.default_rng(seed)
+    for _ in range(12):
+        B = int(rng.choice([5, 33, 100, 257, 1000, 4096, 6000]))
+        k = int(rng.integers(1, min(B, hs.MAX_TOP_K) + 1))
+        N = int(rng.integers(1, 6))
+        lpg = int(rng.choice([1, 1, 2, 4]))
+        L = lpg * int(rng.integers(1, 3))
+        E = int(rng.choice([16, 48, 1152, 4096]))
+        lens = [int(rng.integers(k + 2, 40 * B + 100)) for _ in range(N)]
+        if rng.random() < 0.3:
+            lens[0] = int(rng.integers(80000, 200000))       # page table too large to stage in shared memory
+        S = int(rng.choice([0, 1, 2, 4, 8]))
+        policy = int(rng.choice([hs.POLICY_LRU, hs.POLICY_LRU, hs.POLICY_FIFO, hs.POLICY_RANDOM]))
+        steps = 8
+        w = inputs.Workload("soak", inputs.KIND_DSA_MIX, N, L, lpg, k, B, E, lens, steps, keep=int(k * rng.random()),
+                            recent_window=int(rng.integers(1, 2000)), seed=int(rng.integers(1 << 30)), config_id=77)
+        pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE, ctas_per_request=S, policy=policy, policy_seed=5,
+                    oracle_bytes=E <= 1152)
+        tr = inputs.Trace(w)
+        side = torch.cuda.Stream() if lpg > 1 and rng.random() < 0.7 else None
+        repeat = rng.random() < 0.3
+        try:
+            for _step in range(steps):
+                sel, appended, _ = tr.step()
+                if appended:
+                    pair.append()
+                for layer in range(L):
+                    if layer % lpg == 0:
+                        s = sel[layer // lpg]
+                        if rng.random() < 0.3:
+                            s[rng.random(s.shape) < 0.1] = -1
+                        if repeat and k > 1:
+                            for r in range(N):
+                                s[r, int(rng.integers(k))] = s[r, int(rng.integers(k))]
+                    pair.resolve_and_compare(layer, sel[layer // lpg], side_stream=side)
+                    pair.compare_state(layer)
+            status = pair.gpu.status()
+            assert status == pair.oracle.status and (status & ~hs.STATUS_DUPLICATE) == 0
+            assert int(pair.mism.item()) == 0
+        finally:
+            tr.close()
+            pair.close()
