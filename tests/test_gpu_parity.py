@@ -113,6 +113,14 @@ def test_k_equals_b_all_miss_every_step():
         pair.close()
 
 
+def test_inline_write_through_and_flag_combinations():
+    w = inputs.c1_tiny_dsa()
+    w.steps = 10
+    for flags in (hs.FLAG_INLINE_WRITE_THROUGH, hs.FLAG_INLINE_WRITE_THROUGH | hs.FLAG_NO_PDL | hs.FLAG_PHASE_TIMERS,
+                  hs.FLAG_NO_PDL | hs.FLAG_DEBUG_VALIDATE):
+        run_trace(w, w.steps, flags=flags, pool_every=5)
+
+
 def test_history_capacity_status():
     w = tiny_workload(2, 1, 1, 2, 4, 16, [5, 6], steps=1)     # capacity = len + 2
     pair = Pair(w)
