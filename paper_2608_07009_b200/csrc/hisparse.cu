@@ -13,12 +13,15 @@
 // that every launch is replayable from a CUDA graph.
 //
 // The Resolve kernel (Sec. 3.4, Phases 1-5) runs one thread-block cluster per request.  The cluster's first
-// block does the metadata: it hashes the selected positions into shared memory, probes the position of every
-// slot against that table (coalesced scan of slot_pos), compacts the misses in selection order with
-// ballot/prefix sums, walks the recency order once to split the non-hit slots into the first m (victims) and the
-// rest, and rewrites the order as (untouched ++ victims by slot ++ hits by slot).  After a cluster barrier all
-// blocks of the cluster stream the missing records from pinned host memory into their slots with 16-byte
-// non-coherent loads (Phase 4), so the fetch parallelism does not depend on the number of requests.
+// block does the metadata: it stages the selected row, the recency order and (when it fits) the request's slice of
+// the page table in shared memory with bulk copies, looks every selection up in the page table, marks hit slots in
+// a bitset, compacts the misses in selection order and walks the recency order once (one block scan) to split the
+// non-hit slots into the first m (victims) and the rest, and rewrites the order as (untouched ++ victims by slot
+// ++ hits by slot).  As soon as (position, victim) pairs exist the missing records travel host -> shared memory
+// -> cache slot with cp.async.bulk in both directions (Phase 4); the plan is published to the other blocks of the
+// cluster, which take their share of the records, so the fetch parallelism does not depend on the number of
+// requests.  The launch carries the programmatic-dependent-launch attribute: everything before
+// griddepcontrol.wait depends on nothing an earlier kernel wrote.
 #include "hisparse.h"
 
 #include <cuda_runtime.h>
