@@ -56,6 +56,12 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
 
 #define HISPARSE_FLAG_NO_PDL 16u           /* launch Resolve without programmatic dependent launch             */
 
+#define HISPARSE_FLAG_EAGER_ORDER 32u      /* bring the recency list up to date in every Resolve.  By default a
+                                             Resolve in which nothing missed only stamps its hits (the stamps of
+                                             Sec. 3.2 are the policy's state) and leaves the list behind; the next
+                                             Resolve that needs victims first re-sorts the slots stamped since
+                                             (hisparse_order_lag).  Results are the same either way            */
+
 /* sticky device status bits (hisparse_status) */
 #define HISPARSE_STATUS_OUT_OF_RANGE 1u   /* a selected position was outside [0, len) (and not -1)       */
 #define HISPARSE_STATUS_DUPLICATE 2u      /* a position occurred twice in one row                        */
@@ -187,10 +193,17 @@ int hisparse_clear_status(hisparse_t *h);
 
 /* Copies one (request, layer)'s metadata to host buffers; any pointer may be NULL.  slot_pos [B]
  * (position held by each slot, -1 = empty), last_use [B] (recency stamps), lru_order [B] (slots from
- * least to most recent), pos2slot [capacity[req]] (page table, -1 = host-only).  Synchronises. */
+ * least to most recent as the device holds them: equal to the slots sorted by (last_use, slot) whenever
+ * hisparse_order_lag reports 0), pos2slot [capacity[req]] (page table, -1 = host-only).  Synchronises. */
 int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, uint32_t *last_use,
                         int32_t *lru_order, int32_t *pos2slot, int64_t *len, int64_t *newest,
                         uint32_t *resolves);
+
+/* Number of Resolves of (req, layer's group) that the recency list has not absorbed yet: Resolves in which
+ * nothing missed stamp their hits and leave the list alone; the next Resolve with a miss catches up before it
+ * picks victims, after which the lag is 0 again.  Always 0 with HISPARSE_FLAG_EAGER_ORDER.  The paper keeps
+ * stamps only (Sec. 3.2); the list is this library's own structure.  Synchronises. */
+int hisparse_order_lag(hisparse_t *h, int req, int layer, uint32_t *lag);
 
 /* Checkpoint / resume, the counterparts of hisparse_dump_state (the paper has no such step; its scheduler only
  * releases state).  hisparse_load_appends sets how many records every request has appended so far (lengths =

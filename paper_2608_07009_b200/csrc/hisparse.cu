@@ -69,6 +69,7 @@ struct DevState {
   const int64_t *cap, *init_len, *p2s_off;
   uint8_t *const *host;
   uint32_t *t;
+  uint32_t *order_t;               // [N][G] resolve count up to which `order` is current; null = the list is never left stale
   int32_t *plan_pos, *plan_slot, *plan_n;
   int32_t *anchor_out, *anchor_hits, *anchor_misses;
   int32_t *n_appends;
@@ -442,6 +443,95 @@ __device__ __forceinline__ void cluster_lookups(const int32_t *__restrict__ row,
   cluster_wait();
 }
 
+// Brings a stale recency list up to date.  A resolve without misses leaves the list alone and only stamps its
+// hits, so the list may lag `nsteps` resolves behind the stamps; every slot stamped since (last_use >= thr, all of
+// them hit stamps thr+1, thr+3, ..) belongs behind the untouched slots, ordered by (stamp, slot).  The untouched
+// slots keep their old relative order (one scan, compacted in place); the touched ones are laid out by slot behind
+// them and then sorted by the step that stamped them with one stable in-place split per bit of the step index
+// (no pass at all when a single resolve is outstanding).  s_bits / s_pre: W words each, s_bits is zero on return.
+template <int IPT>
+__device__ __forceinline__ void rebuild_order(const int B, const int W, const uint32_t *__restrict__ last_use,
+                                              const uint32_t thr, const uint32_t nsteps, uint16_t *s_order,
+                                              uint32_t *s_bits, int32_t *s_pre, int *s_warp) {
+  constexpr int T = kThreads;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int sb = 0; sb < B; sb += T) {  // the loop bound is uniform, so every lane takes part in the ballot
+    const int s = sb + tid;
+    const uint32_t word = __ballot_sync(0xffffffffu, s < B && last_use[s] >= thr);
+    if (lane == 0 && (s >> 5) < W) s_bits[s >> 5] = word;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    int run = 0;
+    for (int wb = 0; wb < W; wb += 32) {
+      const int w = wb + lane;
+      const int c = w < W ? __popc(s_bits[w]) : 0;
+      int inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+      }
+      if (w < W) s_pre[w] = run + inc - c;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+  }
+  int n_un;
+  {
+    int slot[IPT];
+    uint32_t un_mask = 0;
+#pragma unroll
+    for (int i = 0; i < IPT; ++i) {
+      const int q = tid * IPT + i;
+      slot[i] = 0;
+      if (q < B) {
+        slot[i] = s_order[q];
+        if (!((s_bits[slot[i] >> 5] >> (slot[i] & 31)) & 1u)) un_mask |= 1u << i;
+      }
+    }
+    int rank = block_scan_excl(__popc(un_mask), s_warp, n_un);  // its barrier also publishes s_pre
+#pragma unroll
+    for (int i = 0; i < IPT; ++i)
+      if ((un_mask >> i) & 1u) s_order[rank++] = (uint16_t)slot[i];  // in place: everything was read before the barrier
+  }
+  for (int s = tid; s < B; s += T) {
+    const int w = s >> 5;
+    const uint32_t bit = 1u << (s & 31), tw = s_bits[w];
+    if (tw & bit) s_order[n_un + s_pre[w] + __popc(tw & (bit - 1u))] = (uint16_t)s;
+  }
+  __syncthreads();
+  for (int i = tid; i < W; i += T) s_bits[i] = 0u;
+  for (uint32_t b = 0; b < 32u && ((nsteps - 1u) >> b) != 0u; ++b) {
+    int slot[IPT];
+    uint32_t valid = 0, one = 0;
+#pragma unroll
+    for (int i = 0; i < IPT; ++i) {
+      const int q = tid * IPT + i;
+      slot[i] = 0;
+      if (q >= n_un && q < B) {
+        slot[i] = s_order[q];
+        valid |= 1u << i;
+        if ((((last_use[slot[i]] - thr) >> 1) >> b) & 1u) one |= 1u << i;
+      }
+    }
+    int n_zero;
+    int z = block_scan_excl(__popc(valid & ~one), s_warp, n_zero);  // zeros before this thread's entries
+#pragma unroll
+    for (int i = 0; i < IPT; ++i)
+      if ((valid >> i) & 1u) {
+        const int idx = tid * IPT + i - n_un;  // place in the touched segment = zeros + ones before it
+        if ((one >> i) & 1u) {
+          s_order[n_un + n_zero + (idx - z)] = (uint16_t)slot[i];
+        } else {
+          s_order[n_un + z] = (uint16_t)slot[i];
+          ++z;
+        }
+      }
+    __syncthreads();
+  }
+  __syncthreads();
+}
+
 // Everything the first block of a cluster does before the fetch can start: Phases 1-3 of Sec. 3.4.
 // IPT = entries of the recency order per thread (B <= IPT * kThreads), KPT = row entries per thread (k <= KPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
 // the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
@@ -455,7 +545,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  const int64_t p2s_off_r, unsigned long long *stamps,
                                                  unsigned char *s_ring, unsigned long long *s_bars,
                                                  const uint32_t t_now, int *s_warp_pre, int16_t *s_got, const int S,
-                                                 int &m, int &n_nonhit, uint32_t &my_status) {
+                                                 const uint32_t order_t, int &m, int &n_nonhit, uint32_t &my_status, bool &fast) {
   constexpr int T = kThreads;
   const int tid = threadIdx.x;
   const int k = d.k, B = d.B, H = d.H;
@@ -538,6 +628,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : coop ? s_got[j] : __ldg(p2s + pos[i]));
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
+  int any_miss = 0;
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
     const int j = tid + i * T;
@@ -557,6 +648,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
         if (atomicOr(&s_hitbits[s >> 5], bit) & bit) my_status |= HISPARSE_STATUS_DUPLICATE;
       } else {
         o = kMiss;
+        any_miss = 1;
         const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)j;
         uint32_t h = hash_pos(p, d.hshift);
         for (uint32_t it = 0; it <= mask; ++it) {
@@ -573,7 +665,15 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     }
     s_out[j] = o;
   }
-  __syncthreads();
+  any_miss = __syncthreads_or(any_miss);
+  if (!any_miss && d.order_t != nullptr) {
+    // Nothing to fetch, no victim to choose: the caller writes the table and stamps the hits, and the recency list
+    // is left as it is (rebuild_order brings it up to date in the next resolve that needs victims).
+    fast = true;
+    m = 0;
+    n_nonhit = 0;
+    return;
+  }
   if (timers && tid == 0) stamps[10] = clock64();
   if (s_misc[0]) {  // rare: every later occurrence of a repeated missing position follows the first one
     for (int j = tid; j < k; j += T) {
@@ -589,7 +689,12 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     }
     __syncthreads();
   }
-  if (timers && tid == 0) { stamps[11] = clock64(); stamps[12] = stamps[11]; }
+  if (timers && tid == 0) stamps[11] = clock64();
+  if (order_t != t_now - 1u) {
+    const uint32_t *last_use = d.last_use + rg * B;
+    rebuild_order<IPT>(B, d.W, last_use, 2u * order_t + 2u, t_now - 1u - order_t, s_order, s_vicbits, s_warp_pre, s_warp);
+  }
+  if (timers && tid == 0) stamps[12] = clock64();
 
   // Phase 3: ONE block scan over packed counts (non-hit slots in recency order | misses in selection order).
   // Thread t owns IPT consecutive entries of the recency order and KPT consecutive row entries.
@@ -750,8 +855,10 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   TmaFetch fetch;
+  fetch.active = false;
   int m = 0, n_nonhit = 0;
   uint32_t t = 0;
+  bool fast = false;  // first block only: no selection missed, the short path below was taken
   if (part != 0) {
     // same test as in resolve_metadata: is this request's page-table slice too large to be staged?
     const int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
@@ -767,13 +874,14 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   if (part == 0) {
     if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
     t = d.t[rg] + 1u;
+    const uint32_t order_t = d.order_t ? d.order_t[rg] : t - 1u;  // resolve count the recency list is current for
     const uint32_t miss_stamp = 2u * t;
     uint32_t my_status = 0;
     const int32_t *row = sel + (int64_t)r * k;
 #define HS_META(IPT, KPT)                                                                                         \
   resolve_metadata<IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
                              s_order, s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t,      \
-                             s_vicpre, s_got, S, m, n_nonhit, my_status)
+                             s_vicpre, s_got, S, order_t, m, n_nonhit, my_status, fast)
     if (k <= 2 * T) {
       if (B <= 4 * T) HS_META(4, 2);
       else if (B <= 8 * T) HS_META(8, 2);
@@ -785,26 +893,62 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     }
 #undef HS_META
     if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
-    // Phase 4 starts here: the first batch of host loads is in flight while the metadata is written back
-    fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
-    fetch.issue();
-    // Phase 5, metadata half: page table, slot array, stamps, plan
-    int32_t *slot_pos = d.slot_pos + rg * B;
-    uint32_t *last_use = d.last_use + rg * B;
-    int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
-    int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
-    for (int i = tid; i < m; i += T) {
-      const int v = s_plan_slot[i];
-      const int32_t p = s_plan_pos[i];
-      const int32_t old = slot_pos[v];
-      if (old >= 0) p2s[old] = -1;
-      slot_pos[v] = p;
-      p2s[p] = (int16_t)v;
-      last_use[v] = miss_stamp;
-      plan_pos_g[i] = p;
-      plan_slot_g[i] = v;
+    if (fast) {
+      // Every valid selection is resident (or the newest record): the slot table, the hit stamps in slot order
+      // (coalesced) and the counters are all there is to write.  The recency list is not touched and
+      // order_t stays behind; under FIFO a hit changes nothing, so the list stays current.
+      int32_t *trow = table + (int64_t)r * k;
+      int32_t *arow = d.anchor_out + rg * k;
+      for (int j = tid; j < k; j += T) {
+        const int32_t o = s_out[j];
+        trow[j] = o < 0 ? -1 : r * (B + 1) + o;
+        if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
+      }
+      int c = 0;
+      for (int w = tid; w < W; w += T) c += __popc(s_hitbits[w]);
+      if (warp * 32 < W) {
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0 && c) atomicAdd(&s_misc[3], c);
+      }
+      if (d.policy != HISPARSE_POLICY_FIFO) {
+        uint32_t *last_use = d.last_use + rg * B;
+        for (int s = tid; s < B; s += T)
+          if ((s_hitbits[s >> 5] >> (s & 31)) & 1u) last_use[s] = 2u * t + 1u;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        const int nhits = s_misc[3] + (s_misc[2] ? 1 : 0);
+        hits_out[r] = nhits;
+        misses_out[r] = 0;
+        d.anchor_hits[rg] = nhits;
+        d.anchor_misses[rg] = 0;
+        d.plan_n[rg] = 0;
+        d.t[rg] = t;
+        if (d.policy == HISPARSE_POLICY_FIFO) d.order_t[rg] = t;
+        if (timers) stamps[4] = global_ns();
+      }
+    } else {
+      // Phase 4 starts here: the first batch of host loads is in flight while the metadata is written back
+      fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
+      fetch.issue();
+      // Phase 5, metadata half: page table, slot array, stamps, plan
+      int32_t *slot_pos = d.slot_pos + rg * B;
+      uint32_t *last_use = d.last_use + rg * B;
+      int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
+      int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
+      for (int i = tid; i < m; i += T) {
+        const int v = s_plan_slot[i];
+        const int32_t p = s_plan_pos[i];
+        const int32_t old = slot_pos[v];
+        if (old >= 0) p2s[old] = -1;
+        slot_pos[v] = p;
+        p2s[p] = (int16_t)v;
+        last_use[v] = miss_stamp;
+        plan_pos_g[i] = p;
+        plan_slot_g[i] = v;
+      }
+      if (tid == 0) d.plan_n[rg] = m;
     }
-    if (tid == 0) d.plan_n[rg] = m;
     if (my_status) atomicOr(d.status, my_status);
     if (S > 1) {
       __threadfence();
@@ -814,7 +958,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
   // The plan is public: the other blocks of the cluster start fetching while this one publishes.
   if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
-  if (part == 0) {
+  if (part == 0 && !fast) {
     uint16_t *order = d.order + rg * B;
     // new order = untouched ++ victims by slot ++ hits by slot: word-level prefix counts, then one pass.
     if (warp == 0) {
@@ -876,6 +1020,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       d.anchor_hits[rg] = nhits;
       d.anchor_misses[rg] = m;
       d.t[rg] = t;
+      if (d.order_t) d.order_t[rg] = t;
     }
     if (timers && tid == 0) stamps[4] = global_ns();
   }
@@ -1045,6 +1190,8 @@ __global__ void validate_kernel(const DevState d, const int g) {
   const int16_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
   for (int i = threadIdx.x; i < d.W; i += blockDim.x) seen[i] = 0u;
   __syncthreads();
+  // a list that lags behind the stamps (resolves without misses) is still a permutation, but not sorted by them
+  const bool current = !d.order_t || d.order_t[rg] == d.t[rg];
   bool bad = false;
   for (int s = threadIdx.x; s < B; s += blockDim.x) {
     const int32_t p = slot_pos[s];
@@ -1061,7 +1208,7 @@ __global__ void validate_kernel(const DevState d, const int g) {
     if (s >= B) { bad = true; continue; }
     const uint32_t old = atomicOr(&seen[s >> 5], 1u << (s & 31));
     bad |= (old >> (s & 31)) & 1u;
-    if (q + 1 < B) {
+    if (q + 1 < B && current) {
       const int s2 = order[q + 1];
       if (s2 < B) {
         const uint32_t a = last_use[s], b = last_use[s2];
@@ -1247,7 +1394,7 @@ int hisparse_device_bytes(const hisparse_config_t *c, size_t *kv_bytes, size_t *
     *meta_bytes = N * G * B * (4 + 4 + 2)          /* slot_pos, last_use, order */
                   + cap_sum * G * 2                 /* page tables */
                   + N * G * k * 4 * 3               /* plan_pos, plan_slot, anchor_out */
-                  + N * G * 4 * 4                   /* t, plan_n, anchor hits / misses */
+                  + N * G * 4 * 5                   /* t, order_t, plan_n, anchor hits / misses */
                   + N * (8 * 3 + 8) + 16;           /* cap, init_len, p2s_off, host pointers, scalars */
   }
   return HISPARSE_OK;
@@ -1345,6 +1492,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRY(dev_alloc(h, &h->d_p2s_off, (size_t)N));
   HS_TRY(dev_alloc(h, &h->d_host, (size_t)N));
   HS_TRY(dev_alloc(h, &d.t, NG));
+  if (!(c->flags & HISPARSE_FLAG_EAGER_ORDER)) HS_TRY(dev_alloc(h, &d.order_t, NG));
   HS_TRY(dev_alloc(h, &d.plan_pos, NG * k));
   HS_TRY(dev_alloc(h, &d.plan_slot, NG * k));
   HS_TRY(dev_alloc(h, &d.plan_n, NG));
@@ -1371,6 +1519,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRYC(cudaMemset(d.last_use, 0, NG * B * 4));
   HS_TRYC(cudaMemset(d.pos2slot, 0xff, (size_t)h->p2s_total * 2));
   HS_TRYC(cudaMemset(d.t, 0, NG * 4));
+  if (d.order_t) HS_TRYC(cudaMemset(d.order_t, 0, NG * 4));
   HS_TRYC(cudaMemset(d.plan_n, 0, NG * 4));
   HS_TRYC(cudaMemset(d.anchor_out, 0xff, NG * k * 4));
   HS_TRYC(cudaMemset(d.anchor_hits, 0, NG * 4));
@@ -1608,6 +1757,20 @@ int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, ui
   return HISPARSE_OK;
 }
 
+int hisparse_order_lag(hisparse_t *h, int req, int layer, uint32_t *lag) {
+  if (!h || req < 0 || req >= h->d.N || layer < 0 || layer >= h->d.L || !lag) return HISPARSE_EINVAL;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  *lag = 0;
+  if (!h->d.order_t) return HISPARSE_OK;
+  const int64_t rg = (int64_t)req * h->d.G + layer / h->d.lpg;
+  uint32_t t = 0, ot = 0;
+  HS_CUDA(cudaMemcpy(&t, h->d.t + rg, 4, cudaMemcpyDeviceToHost));
+  HS_CUDA(cudaMemcpy(&ot, h->d.order_t + rg, 4, cudaMemcpyDeviceToHost));
+  *lag = t - ot;
+  return HISPARSE_OK;
+}
+
 int hisparse_load_state(hisparse_t *h, int req, int layer, const int32_t *slot_pos, const uint32_t *last_use,
                         uint32_t resolves) {
   if (!h || req < 0 || req >= h->d.N || layer < 0 || layer >= h->d.L || !slot_pos || !last_use) return HISPARSE_EINVAL;
@@ -1635,6 +1798,7 @@ int hisparse_load_state(hisparse_t *h, int req, int layer, const int32_t *slot_p
   HS_CUDA(cudaMemcpy(h->d.order + rg * B, order.data(), (size_t)B * 2, cudaMemcpyHostToDevice));
   HS_CUDA(cudaMemcpy(h->d.pos2slot + h->p2s_off[req] + (int64_t)g * cap, p2s.data(), (size_t)cap * 2, cudaMemcpyHostToDevice));
   HS_CUDA(cudaMemcpy(h->d.t + rg, &resolves, 4, cudaMemcpyHostToDevice));
+  if (h->d.order_t) HS_CUDA(cudaMemcpy(h->d.order_t + rg, &resolves, 4, cudaMemcpyHostToDevice));  // the list is current
   const int32_t zero = 0;
   HS_CUDA(cudaMemcpy(h->d.plan_n + rg, &zero, 4, cudaMemcpyHostToDevice));
   // the host history is authoritative: refill every layer of the group from it (resident records + newest record)
@@ -1846,7 +2010,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   const int optin = g_noalloc_optin[dev];
   lock.unlock();
 
-  DevState d{};
+  DevState d{};  // order_t stays null: the caller's recency list is brought up to date by every call
   d.N = N; d.L = 1; d.lpg = 1; d.G = 1; d.B = B; d.k = k;
   d.H = hash_size(k); d.W = (B + 31) / 32;
   d.hshift = 32;

@@ -17,6 +17,7 @@ from . import build as _build
 OK, EINVAL, ENOTPINNED, ENOMEM, ECUDA, ESTATE, ETOOBIG = 0, -1, -2, -3, -4, -5, -6
 NOALLOC_MAX_REQUESTS, NOALLOC_MAX_SELECTIONS = 1024, 65536
 FLAG_SKIP_IO, FLAG_DEBUG_VALIDATE, FLAG_INLINE_WRITE_THROUGH, FLAG_PHASE_TIMERS, FLAG_NO_PDL = 1, 2, 4, 8, 16
+FLAG_EAGER_ORDER = 32
 STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, STATUS_CAPACITY, STATUS_INCONSISTENT, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 MAX_CACHE_SLOTS, MAX_TOP_K = 16384, 4096
 POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2
@@ -24,7 +25,7 @@ POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2
 EXPORTS = [
     "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch", "hisparse_prefetch_hint",
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
-    "hisparse_clear_status", "hisparse_dump_state", "hisparse_load_state", "hisparse_load_appends", "hisparse_dump_plan", "hisparse_device_bytes",
+    "hisparse_clear_status", "hisparse_dump_state", "hisparse_order_lag", "hisparse_load_state", "hisparse_load_appends", "hisparse_dump_plan", "hisparse_device_bytes",
     "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_selftest_wait_timeout", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
     "hisparse_scatter_read_probe", "hisparse_resolve_noalloc", "hisparse_strerror", "hisparse_last_cuda_error",
 ]
@@ -89,6 +90,7 @@ def lib() -> ctypes.CDLL:
             "hisparse_clear_status": ([vp], i32),
             "hisparse_dump_state": ([vp, i32, i32, vp, vp, vp, vp, P(i64), P(i64), P(u32)], i32),
             "hisparse_load_state": ([vp, i32, i32, vp, vp, u32], i32),
+            "hisparse_order_lag": ([vp, i32, i32, P(u32)], i32),
             "hisparse_load_appends": ([vp, ctypes.c_int32], i32),
             "hisparse_dump_plan": ([vp, i32, i32, vp, vp, P(ctypes.c_int32)], i32),
             "hisparse_device_bytes": ([P(Config), P(sz), P(sz)], i32),
@@ -311,6 +313,13 @@ class HiSparse:
         assert sp.size == self.B and lu.size == self.B
         _check(lib().hisparse_load_state(self._h, req, layer, sp.ctypes.data, lu.ctypes.data, resolves),
                "hisparse_load_state")
+
+    def order_lag(self, req: int, layer: int) -> int:
+        """Resolves of (req, layer's group) the recency list has not absorbed yet (0 = dump_state's lru_order is the
+        slots sorted by (last_use, slot))."""
+        lag = ctypes.c_uint32()
+        _check(lib().hisparse_order_lag(self._h, req, layer, ctypes.byref(lag)), "hisparse_order_lag")
+        return int(lag.value)
 
     def dump_plan(self, req: int, layer: int):
         pos = np.empty(self.k, dtype=np.int32)

@@ -9,6 +9,21 @@ from oracle import Oracle, FLAG_NO_BYTES
 from paper_2608_07009_b200 import HiSparse, HostHistory, inputs
 
 
+def check_recency_list(order, last_use, lag, resolves):
+    """The recency list the kernels keep is the slots sorted by (stamp, slot) whenever it is current (lag 0).  After
+    `lag` resolves without misses it is still a permutation, and the slots not stamped since (stamp below the first
+    stamp of those resolves) still stand in it in (stamp, slot) order."""
+    B = len(last_use)
+    want = np.lexsort((np.arange(B), last_use))
+    if lag == 0:
+        assert np.array_equal(order, want)
+        return
+    assert lag <= resolves
+    assert np.array_equal(np.sort(order), np.arange(B))
+    thr = 2 * (resolves - lag) + 2
+    assert np.array_equal(order[last_use[order] < thr], want[last_use[want] < thr])
+
+
 class Pair:
     """One CUDA handle and one oracle over separate copies of the same host histories."""
 
@@ -82,8 +97,7 @@ class Pair:
             assert np.array_equal(st["pos2slot"], self.oracle.pos2slot(r, layer)), (r, layer)
             assert st["len"] == self.oracle.length(r) and st["newest"] == self.oracle.newest(r)
             assert st["resolves"] == self.oracle.steps(r, layer)
-            # the recency list the kernels keep is exactly the slots sorted by (stamp, slot)
-            assert np.array_equal(st["lru_order"], np.lexsort((np.arange(w.cache_slots), lu)))
+            check_recency_list(st["lru_order"], lu, self.gpu.order_lag(r, layer), st["resolves"])
             pp, ps = self.gpu.dump_plan(r, layer)
             op, os_ = self.oracle.plan(r, layer)
             assert np.array_equal(pp, op) and np.array_equal(ps, os_)

@@ -18,6 +18,7 @@ import torch
 
 from oracle import Oracle, FLAG_NO_BYTES
 from paper_2608_07009_b200 import HiSparse, HostHistory, HiSparseError, inputs, hisparse as hs
+from gpu_harness import check_recency_list
 
 pytestmark = pytest.mark.gpu
 REDUCED = os.environ.get("HISPARSE_REDUCED_LAYERS", "0") == "1"
@@ -91,7 +92,7 @@ def run_full(w, steps, sample_pairs, use_prefetch=False):
                     lu = orc.last_use(r, layer)
                     assert np.array_equal(st["last_use"], lu)
                     assert np.array_equal(st["pos2slot"], orc.pos2slot(r, layer))
-                    assert np.array_equal(st["lru_order"], np.lexsort((np.arange(B), lu)))
+                    check_recency_list(st["lru_order"], lu, gpu.order_lag(r, layer), st["resolves"])
                     assert st["len"] == orc.length(r) and st["newest"] == orc.newest(r)
                     pp, ps = gpu.dump_plan(r, layer)
                     op, os_ = orc.plan(r, layer)

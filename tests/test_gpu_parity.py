@@ -243,6 +243,119 @@ def test_policies_c2_shape_and_groups(policy):
     run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=7)
 
 
+# ------------------------------------------------------------------ recency list left behind by hit-only resolves
+
+def _hit_only_rows(rng, pair, k, newest_too, layer=0):
+    """A row per request drawn from what is resident (so that nothing misses), padded with -1."""
+    rows = []
+    for r in range(pair.w.num_requests):
+        res = pair.oracle.slot_pos(r, layer)
+        res = res[res >= 0]
+        n = int(rng.integers(0, min(k, len(res)) + 1))
+        row = rng.choice(res, size=n, replace=False).astype(np.int32)
+        if newest_too and pair.oracle.newest(r) >= 0 and n < k:
+            row = np.append(row, np.int32(pair.oracle.newest(r)))
+        row = np.concatenate([row, np.full(k - len(row), -1, dtype=np.int32)])
+        rows.append(rng.permutation(row))
+    return np.stack(rows)
+
+
+@pytest.mark.parametrize("policy", [hs.POLICY_LRU, hs.POLICY_FIFO, hs.POLICY_RANDOM])
+@pytest.mark.parametrize("B,k,S", [(4, 2, 1), (12, 5, 2), (40, 17, 1), (300, 130, 4), (5000, 2100, 1)])
+def test_list_catches_up_after_hit_only_runs(policy, B, k, S):
+    """Runs of 1..9 resolves in which nothing misses (the list is left behind and only stamps are written), each
+    followed by resolves with misses (the list is re-sorted before victims are taken): everything still equals the
+    oracle, and the list's lag is what the schedule says."""
+    rng = np.random.default_rng(1000 * policy + B)
+    w = tiny_workload(2, 1, 1, k, B, 32, [3 * B + 7, 2 * B + 3])
+    pair = Pair(w, policy=policy, policy_seed=5, flags=hs.FLAG_DEBUG_VALIDATE, ctas_per_request=S)
+    try:
+        for run in (1, 2, 3, 1, 5, 9, 2):
+            for _ in range(2):   # resolves with misses
+                pair.append()
+                rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0] for r in range(2)])
+                _, _, m = pair.resolve_and_compare(0, rows)
+                pair.compare_state(0)
+                for r in range(2):
+                    assert pair.gpu.order_lag(r, 0) == 0 or m[r] == 0
+            for i in range(run):
+                _, _, m = pair.resolve_and_compare(0, _hit_only_rows(rng, pair, k, newest_too=i % 2 == 1))
+                assert int(m.sum()) == 0
+                pair.compare_state(0)
+                if policy != hs.POLICY_FIFO:
+                    assert all(pair.gpu.order_lag(r, 0) >= i + 1 for r in range(2))
+                else:
+                    assert all(pair.gpu.order_lag(r, 0) == 0 for r in range(2))
+        pair.finish()
+    finally:
+        pair.close()
+
+
+def test_eager_list_flag_gives_the_same_results_and_never_lags():
+    rng = np.random.default_rng(77)
+    B, k = 300, 130
+    w = tiny_workload(2, 1, 1, k, B, 32, [3 * B + 7, 2 * B + 3])
+    pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE | hs.FLAG_EAGER_ORDER)
+    try:
+        for step in range(12):
+            if step % 3 == 0:
+                rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0] for r in range(2)])
+            else:
+                rows = _hit_only_rows(rng, pair, k, newest_too=False)
+            pair.resolve_and_compare(0, rows)
+            pair.compare_state(0)
+            assert all(pair.gpu.order_lag(r, 0) == 0 for r in range(2))
+        pair.finish()
+    finally:
+        pair.close()
+
+
+def test_hit_only_resolves_in_shared_groups_and_after_resume():
+    """Groups of layers: a hit-only anchor resolve still hands its table to the shared layers and an empty plan to
+    the prefetch.  A state dumped while the list lags resumes exactly (load_state rebuilds the list)."""
+    rng = np.random.default_rng(5)
+    B, k = 64, 20
+    w = tiny_workload(2, 4, 2, k, B, 48, [200, 150])
+    pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE)
+    side = torch.cuda.Stream()
+    try:
+        for step in range(10):
+            pair.append()
+            for g in range(2):
+                if step % 4 == 0:
+                    rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0] for r in range(2)])
+                else:
+                    rows = _hit_only_rows(rng, pair, k, newest_too=step % 2 == 1, layer=2 * g)
+                for layer in (2 * g, 2 * g + 1):
+                    pair.resolve_and_compare(layer, rows, side_stream=side)
+                    pair.compare_state(layer)
+        assert pair.gpu.order_lag(0, 0) > 0
+        # resume into a second handle from the dumped stamps while the list lags
+        st = [[pair.gpu.dump_state(r, 2 * g) for g in range(2)] for r in range(2)]
+        appends = st[0][0]["len"] - w.init_len[0]
+        other = HiSparse(2, 4, 2, B, k, 48, w.capacity, w.init_len, pair.hist_gpu, flags=hs.FLAG_DEBUG_VALIDATE)
+        try:
+            other.load_appends(appends)
+            for r in range(2):
+                for g in range(2):
+                    other.load_state(r, 2 * g, st[r][g]["slot_pos"], st[r][g]["last_use"], st[r][g]["resolves"])
+                    assert other.order_lag(r, 2 * g) == 0
+            rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0] for r in range(2)])
+            rows_d = torch.from_numpy(rows).to(pair.dev)
+            tab_a, h_a, m_a = pair.gpu.resolve(0, rows_d)
+            tab_b, h_b, m_b = other.resolve(0, rows_d)
+            assert torch.equal(tab_a, tab_b) and torch.equal(h_a, h_b) and torch.equal(m_a, m_b)
+            for r in range(2):
+                a, b = pair.gpu.dump_state(r, 0), other.dump_state(r, 0)
+                for key in ("slot_pos", "last_use", "lru_order", "pos2slot"):
+                    assert np.array_equal(a[key], b[key]), key
+            assert other.status() == 0
+        finally:
+            other.close()
+    finally:
+        pair.close()
+
+
 # ------------------------------------------------------------------ speculative hints
 
 def test_speculative_hint_is_a_discarded_resolve():
