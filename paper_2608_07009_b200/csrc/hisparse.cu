@@ -854,6 +854,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a), "r"((uint32_t)n) : "memory");
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (part != 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   TmaFetch fetch;
   fetch.active = false;
   int m = 0, n_nonhit = 0;
@@ -894,6 +895,10 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
 #undef HS_META
     if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
     if (fast) {
+      // nothing to fetch: let whatever follows in the stream start its prologue now (measured: with a fetch ahead,
+      // releasing the dependents before the first loads are issued costs the fetch about 2 us, so that path
+      // releases them only once its metadata is written back)
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
       // Every valid selection is resident (or the newest record): the slot table, the hit stamps in slot order
       // (coalesced) and the counters are all there is to write.  The recency list is not touched and
       // order_t stays behind; under FIFO a hit changes nothing, so the list stays current.
