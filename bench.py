@@ -56,6 +56,8 @@ def parse_args():
                     help="speculative prefetch: layer l's selection is given to layer l+1 as a hint (side stream)")
     ap.add_argument("--no-pdl", action="store_true", help="launch Resolve without programmatic dependent launch")
     ap.add_argument("--no-all-hit", action="store_true", help="skip the scaled all-hit HBM point")
+    ap.add_argument("--wide-blocks", action="store_true", help="1024-thread blocks even when the grid takes several waves")
+    ap.add_argument("--eager-order", action="store_true", help="update the recency list in every resolve")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-requests", type=int, default=8)
     ap.add_argument("--cpu-sample-steps", type=int, default=200, help="oracle steps timed by the cpu_baseline leg")
@@ -336,7 +338,8 @@ def run_ours(args):
     for r, h in enumerate(hist):
         inputs.fill_history(h.ptr, r, L, cap[r], 0, w.init_len[r], E, w.seed)
     flags = (hs.FLAG_SKIP_IO if args.skip_io else 0) | (hs.FLAG_PHASE_TIMERS if args.phases else 0) \
-        | (hs.FLAG_NO_PDL if args.no_pdl else 0)
+        | (hs.FLAG_NO_PDL if args.no_pdl else 0) | (hs.FLAG_WIDE_BLOCKS if args.wide_blocks else 0) \
+        | (hs.FLAG_EAGER_ORDER if args.eager_order else 0)
     gpu = hs.HiSparse(N, L, lpg, B, k, E, cap, w.init_len, hist, device=local, flags=flags,
                       ctas_per_request=args.ctas_per_request)
     geo = gpu.launch_geometry()

@@ -62,6 +62,13 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
                                              Resolve that needs victims first re-sorts the slots stamped since
                                              (hisparse_order_lag).  Results are the same either way            */
 
+#define HISPARSE_FLAG_WIDE_BLOCKS 64u       /* always one 1024-thread block per SM.  By default a handle whose grid
+                                             takes several waves (more blocks than SMs) runs two 512-thread blocks
+                                             per SM when B <= 8192 and k <= 2048 (hisparse_launch_geometry)       */
+
+#define HISPARSE_FLAG_NARROW_BLOCKS 128u    /* always 512-thread blocks; EINVAL when the shape does not allow them
+                                             (or together with WIDE_BLOCKS).  Results do not depend on the block size */
+
 /* sticky device status bits (hisparse_status) */
 #define HISPARSE_STATUS_OUT_OF_RANGE 1u   /* a selected position was outside [0, len) (and not -1)       */
 #define HISPARSE_STATUS_DUPLICATE 2u      /* a position occurred twice in one row                        */

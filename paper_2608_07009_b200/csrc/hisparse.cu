@@ -47,7 +47,8 @@ thread_local int g_last_cuda_error = 0;
     }                                                   \
   } while (0)
 
-constexpr int kThreads = 1024;       // threads per block of the resolve / replay kernels
+constexpr int kThreads = 1024;       // most threads per block of the resolve / replay kernels (one block per SM)
+constexpr int kThreadsSmall = 512;   // block size when the grid takes several waves: two blocks share an SM
 constexpr int kFetchUnroll = 4;      // 16-byte host loads in flight per thread (probe kernel)
 constexpr int kBarBytes = (kThreads + 2) * 8;  // one mbarrier per thread for the fetch ring + one for staging
 constexpr int32_t kMiss = -2;        // s_out marker: valid selection, not (yet) found resident
@@ -415,16 +416,17 @@ __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.w
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_relaxed() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
 
+template <int T>
 __device__ __forceinline__ void cluster_lookups(const int32_t *__restrict__ row, const int16_t *__restrict__ p2s,
                                                 const int k, const int64_t len, const int part, const int S,
                                                 int16_t *s_got) {
-  constexpr int kMaxPer = (HISPARSE_MAX_TOP_K / 2 + kThreads - 1) / kThreads;  // S >= 2, so a block's share <= k/2
+  constexpr int kMaxPer = (HISPARSE_MAX_TOP_K / 2 + T - 1) / T;  // S >= 2, so a block's share <= k/2
   const int chunk = (k + S - 1) / S;
   const int lo = part * chunk, hi = lo + chunk < k ? lo + chunk : k;
   int16_t v[kMaxPer];
 #pragma unroll
   for (int i = 0; i < kMaxPer; ++i) {
-    const int j = lo + (int)threadIdx.x + i * kThreads;
+    const int j = lo + (int)threadIdx.x + i * T;
     v[i] = -1;
     if (j < hi) {
       const int32_t p = __ldg(row + j);
@@ -436,7 +438,7 @@ __device__ __forceinline__ void cluster_lookups(const int32_t *__restrict__ row,
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote_base) : "r"(smem_u32(s_got)), "r"(0));
 #pragma unroll
   for (int i = 0; i < kMaxPer; ++i) {
-    const int j = lo + (int)threadIdx.x + i * kThreads;
+    const int j = lo + (int)threadIdx.x + i * T;
     if (j < hi) asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(remote_base + 2u * (uint32_t)j), "h"(v[i]) : "memory");
   }
   cluster_arrive();  // phase B
@@ -449,11 +451,10 @@ __device__ __forceinline__ void cluster_lookups(const int32_t *__restrict__ row,
 // slots keep their old relative order (one scan, compacted in place); the touched ones are laid out by slot behind
 // them and then sorted by the step that stamped them with one stable in-place split per bit of the step index
 // (no pass at all when a single resolve is outstanding).  s_bits / s_pre: W words each, s_bits is zero on return.
-template <int IPT>
+template <int T, int IPT>
 __device__ __forceinline__ void rebuild_order(const int B, const int W, const uint32_t *__restrict__ last_use,
                                               const uint32_t thr, const uint32_t nsteps, uint16_t *s_order,
                                               uint32_t *s_bits, int32_t *s_pre, int *s_warp) {
-  constexpr int T = kThreads;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int sb = 0; sb < B; sb += T) {  // the loop bound is uniform, so every lane takes part in the ballot
     const int s = sb + tid;
@@ -536,7 +537,7 @@ __device__ __forceinline__ void rebuild_order(const int B, const int W, const ui
 // IPT = entries of the recency order per thread (B <= IPT * kThreads), KPT = row entries per thread (k <= KPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
 // the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
 // the untouched slots compacted at its front, and s_hitbits / s_vicbits the per-slot marks.
-template <int IPT, int KPT>
+template <int T, int IPT, int KPT>
 __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r, const int64_t rg, const int32_t *row,
                                                  int32_t *s_sel, int32_t *s_out, int32_t *s_plan_pos,
                                                  int32_t *s_plan_slot, unsigned long long *s_tab, uint32_t *s_hitbits,
@@ -546,7 +547,6 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  unsigned char *s_ring, unsigned long long *s_bars,
                                                  const uint32_t t_now, int *s_warp_pre, int16_t *s_got, const int S,
                                                  const uint32_t order_t, int &m, int &n_nonhit, uint32_t &my_status, bool &fast) {
-  constexpr int T = kThreads;
   const int tid = threadIdx.x;
   const int k = d.k, B = d.B, H = d.H;
   const uint32_t mask = (uint32_t)(H - 1);
@@ -584,7 +584,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                  ::"r"(smem_u32(s_order)), "l"(order_g), "r"((uint32_t)B * 2u), "r"(stage_bar) : "memory");
   if (staged && tid >= 64 && (tid & 31) == 0) {
     constexpr int kPiece = 16384;
-    for (int64_t o = (int64_t)((tid >> 5) - 2) * kPiece; o < stage_bytes; o += (int64_t)(kThreads / 32 - 2) * kPiece) {
+    for (int64_t o = (int64_t)((tid >> 5) - 2) * kPiece; o < stage_bytes; o += (int64_t)(T / 32 - 2) * kPiece) {
       const uint32_t n = (uint32_t)(stage_bytes - o < kPiece ? stage_bytes - o : kPiece);
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                    ::"r"(smem_u32(s_ring) + (uint32_t)o), "l"((const char *)p2s_aligned + o), "r"(n), "r"(stage_bar) : "memory");
@@ -611,7 +611,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   __syncthreads();
   if (timers && tid == 0) stamps[9] = clock64();
   const int16_t *s_p2s = reinterpret_cast<const int16_t *>(s_ring) + lead;
-  if (coop) cluster_lookups(row, p2s, k, len, 0, S, s_got);
+  if (coop) cluster_lookups<T>(row, p2s, k, len, 0, S, s_got);
 
   // Phase 2: hit detection through the page table (position -> slot): all of a thread's lookups are issued
   // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
@@ -692,7 +692,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   if (timers && tid == 0) stamps[11] = clock64();
   if (order_t != t_now - 1u) {
     const uint32_t *last_use = d.last_use + rg * B;
-    rebuild_order<IPT>(B, d.W, last_use, 2u * order_t + 2u, t_now - 1u - order_t, s_order, s_vicbits, s_warp_pre, s_warp);
+    rebuild_order<T, IPT>(B, d.W, last_use, 2u * order_t + 2u, t_now - 1u - order_t, s_order, s_vicbits, s_warp_pre, s_warp);
   }
   if (timers && tid == 0) stamps[12] = clock64();
 
@@ -801,13 +801,13 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
   if (timers && tid == 0) stamps[14] = clock64();
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+template <int T>
+__global__ void __launch_bounds__(T, kThreads / T)
 resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ sel, int32_t *__restrict__ table,
                int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out, const int S) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int s_warp[32];
   __shared__ int s_misc[4];  // [0] a missing position was selected twice  [2] the newest position was selected
-  constexpr int T = kThreads;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x / S, part = blockIdx.x - r * S;
   const int g = layer / d.lpg;
@@ -869,7 +869,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       const int64_t na = *(volatile int32_t *)d.n_appends;
       const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
       cluster_arrive_relaxed();  // phase A
-      cluster_lookups(sel + (int64_t)r * k, p2s, k, len, part, S, s_got);
+      cluster_lookups<T>(sel + (int64_t)r * k, p2s, k, len, part, S, s_got);
     }
   }
   if (part == 0) {
@@ -880,17 +880,22 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     uint32_t my_status = 0;
     const int32_t *row = sel + (int64_t)r * k;
 #define HS_META(IPT, KPT)                                                                                         \
-  resolve_metadata<IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
+  resolve_metadata<T, IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
                              s_order, s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t,      \
                              s_vicpre, s_got, S, order_t, m, n_nonhit, my_status, fast)
-    if (k <= 2 * T) {
-      if (B <= 4 * T) HS_META(4, 2);
-      else if (B <= 8 * T) HS_META(8, 2);
-      else HS_META(16, 2);
-    } else {
-      if (B <= 4 * T) HS_META(4, kSelPerThread);
-      else if (B <= 8 * T) HS_META(8, kSelPerThread);
-      else HS_META(16, kSelPerThread);
+    if constexpr (T == kThreads) {
+      if (k <= 2 * T) {
+        if (B <= 4 * T) HS_META(4, 2);
+        else if (B <= 8 * T) HS_META(8, 2);
+        else HS_META(16, 2);
+      } else {
+        if (B <= 4 * T) HS_META(4, kSelPerThread);
+        else if (B <= 8 * T) HS_META(8, kSelPerThread);
+        else HS_META(16, kSelPerThread);
+      }
+    } else {  // the small block is only chosen for B <= 16 T and k <= 4 T
+      if (B <= 8 * T) HS_META(8, 4);
+      else HS_META(16, 4);
     }
 #undef HS_META
     if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
@@ -1341,6 +1346,11 @@ size_t resolve_smem_bytes(int B, int k) {
 
 cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
 
+const void *resolve_kernel_of(int threads) {
+  return threads == kThreadsSmall ? reinterpret_cast<const void *>(&resolve_kernel<kThreadsSmall>)
+                                  : reinterpret_cast<const void *>(&resolve_kernel<kThreads>);
+}
+
 int launch_resolve(hisparse *h, int layer, const int32_t *sel, int32_t *table, int32_t *hits, int32_t *misses,
                    cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
@@ -1357,7 +1367,10 @@ int launch_resolve(hisparse *h, int layer, const int32_t *sel, int32_t *table, i
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (h->d.flags & HISPARSE_FLAG_NO_PDL) ? 1 : 2;
-  HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel, h->d, layer, sel, table, hits, misses, h->S));
+  if (h->T == kThreadsSmall)
+    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreadsSmall>, h->d, layer, sel, table, hits, misses, h->S));
+  else
+    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreads>, h->d, layer, sel, table, hits, misses, h->S));
   return HISPARSE_OK;
 }
 
@@ -1443,22 +1456,41 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   for (int r = 0; r < N; ++r) { h->p2s_off[r] = off; off += h->cap[r] * G; }
   h->p2s_total = off;
 
-  int max_optin = 0;
+  int max_optin = 0, smem_per_sm = 0, sm_count = 0;
   if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  if (cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  // Block size.  One 1024-thread block per SM gives a request the whole SM and all of its shared memory for the
+  // fetch ring.  When the grid takes several waves anyway (more blocks than SMs), two 512-thread blocks per SM hide
+  // each other's dependent trips to memory; each then gets half of the SM's shared memory.
+  int want = c->ctas_per_request;
+  if (!want) {
+    want = 1;
+    while (want < 8 && N * want < 32) want <<= 1;
+  }
+  d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
+  const int64_t budget_small = smem_per_sm / 2 - 1024 - 256;   // per block: 1 KB reserved by the system, static arrays
+  const bool fits_small = B <= 16 * kThreadsSmall && k <= 4 * kThreadsSmall &&
+                          budget_small - d.meta_smem - kBarBytes >= std::min<int64_t>(d.E, 8192) * 8;
+  if ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) && ((c->flags & HISPARSE_FLAG_WIDE_BLOCKS) || !fits_small)) return fail(HISPARSE_EINVAL);
+  const bool small = fits_small && !(c->flags & HISPARSE_FLAG_WIDE_BLOCKS) &&
+                     ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) || (int64_t)N * want > sm_count);
+  h->T = small ? kThreadsSmall : kThreads;
+  const int64_t budget = small ? budget_small : (int64_t)max_optin - 1024;
   // shared memory: metadata arrays, one mbarrier per thread, then the staging ring of the fetch pipeline,
   // which takes whatever is left (pieces of at most 8 KB; at least one piece must fit)
-  d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
-  const int64_t ring_room = (int64_t)max_optin - 1024 - d.meta_smem - kBarBytes;
+  const int64_t ring_room = budget - d.meta_smem - kBarBytes;
   if (ring_room < 16) return fail(HISPARSE_EINVAL);
   d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
   const int slots = (int)(ring_room / d.io_chunk);
-  d.io_threads = std::min(slots, kThreads);
+  d.io_threads = std::min(slots, h->T);
   d.io_depth = std::min(slots / d.io_threads, 8);
   d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
   d.io_ppr = (int)((d.E + d.io_chunk - 1) / d.io_chunk);
   h->resolve_smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
   h->replay_smem = h->resolve_smem;   // same offsets, so that both kernels share the pipeline's geometry
-  if (cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  const void *kern = resolve_kernel_of(h->T);
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaFuncSetAttribute(replay_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
 
   // Blocks per request: enough of them that about 32 blocks pull on the host link together (measured: fewer
@@ -1467,20 +1499,18 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   if (c->ctas_per_request) {
     h->S = c->ctas_per_request;
   } else {
-    int want = 1;
-    while (want < 8 && N * want < 32) want <<= 1;
     h->S = 1;
     for (int s = want; s > 1; s >>= 1) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)(N * s));
-      cfg.blockDim = dim3(kThreads);
+      cfg.blockDim = dim3((unsigned)h->T);
       cfg.dynamicSmemBytes = h->resolve_smem;
       cudaLaunchAttribute attr[1];
       attr[0].id = cudaLaunchAttributeClusterDimension;
       attr[0].val.clusterDim.x = (unsigned)s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
       cfg.attrs = attr; cfg.numAttrs = 1;
       int nclusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&nclusters, resolve_kernel, &cfg) == cudaSuccess && nclusters >= N) { h->S = s; break; }
+      if (cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg) == cudaSuccess && nclusters >= N) { h->S = s; break; }
       cudaGetLastError();
     }
   }
@@ -2007,7 +2037,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
     HS_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
     int optin = 0;
     HS_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    HS_CUDA(cudaFuncSetAttribute(resolve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 1024));
+    HS_CUDA(cudaFuncSetAttribute(resolve_kernel<kThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 1024));
     g_noalloc_optin[dev] = optin;
     g_noalloc_ptr[dev] = static_cast<unsigned char *>(p);
   }
@@ -2063,7 +2093,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel, d, 0, sel_dev, slot_table_dev, hits_dev, misses_dev, S));
+  HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreads>, d, 0, sel_dev, slot_table_dev, hits_dev, misses_dev, S));
   return HISPARSE_OK;
 }
 

@@ -17,7 +17,7 @@ from . import build as _build
 OK, EINVAL, ENOTPINNED, ENOMEM, ECUDA, ESTATE, ETOOBIG = 0, -1, -2, -3, -4, -5, -6
 NOALLOC_MAX_REQUESTS, NOALLOC_MAX_SELECTIONS = 1024, 65536
 FLAG_SKIP_IO, FLAG_DEBUG_VALIDATE, FLAG_INLINE_WRITE_THROUGH, FLAG_PHASE_TIMERS, FLAG_NO_PDL = 1, 2, 4, 8, 16
-FLAG_EAGER_ORDER = 32
+FLAG_EAGER_ORDER, FLAG_WIDE_BLOCKS, FLAG_NARROW_BLOCKS = 32, 64, 128
 STATUS_OUT_OF_RANGE, STATUS_DUPLICATE, STATUS_CAPACITY, STATUS_INCONSISTENT, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 MAX_CACHE_SLOTS, MAX_TOP_K = 16384, 4096
 POLICY_LRU, POLICY_FIFO, POLICY_RANDOM = 0, 1, 2

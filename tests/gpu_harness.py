@@ -35,9 +35,14 @@ class Pair:
         self.hist_gpu = [HostHistory(w.num_layers, cap[r], w.entry_bytes) for r in range(w.num_requests)]
         for r, h in enumerate(self.hist_gpu):
             inputs.fill_history(h.ptr, r, w.num_layers, cap[r], 0, il[r], w.entry_bytes, w.seed)
-        self.gpu = HiSparse(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k, w.entry_bytes,
-                            cap, il, self.hist_gpu, device=device, flags=flags, ctas_per_request=ctas_per_request,
-                            policy=policy, policy_seed=policy_seed)
+        try:
+            self.gpu = HiSparse(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k, w.entry_bytes,
+                                cap, il, self.hist_gpu, device=device, flags=flags, ctas_per_request=ctas_per_request,
+                                policy=policy, policy_seed=policy_seed)
+        except Exception:
+            for h in self.hist_gpu:
+                h.free()
+            raise
         self.oracle_bytes = oracle_bytes
         if oracle_bytes:
             self.hist_cpu = [inputs.new_history(w, r) for r in range(w.num_requests)]

@@ -243,6 +243,85 @@ def test_policies_c2_shape_and_groups(policy):
     run_trace(w, w.steps, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=7)
 
 
+# ------------------------------------------------------------------ 512-thread blocks (two per SM)
+
+NARROW = hs.FLAG_NARROW_BLOCKS | hs.FLAG_DEBUG_VALIDATE
+
+
+@pytest.mark.parametrize("B", [1, 3, 8, 12])
+def test_narrow_blocks_tiny_matrix(B):
+    rng = np.random.default_rng(40 + B)
+    for k in range(1, B + 1):
+        w = tiny_workload(2, 1, 1, k, B, 32, [2 * B + 3, 3 * B + 1])
+        pair = Pair(w, flags=NARROW)
+        try:
+            assert pair.gpu.launch_geometry()["threads"] == 512
+            for step in range(12):
+                if step % 3 == 2:
+                    pair.append()
+                rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.15)[0] for r in range(2)])
+                pair.resolve_and_compare(0, rows)
+                pair.compare_state(0)
+            pair.finish()
+        finally:
+            pair.close()
+
+
+@pytest.mark.parametrize("S", [1, 2, 4, 8])
+def test_narrow_blocks_c2_shape(S):
+    w = inputs.c2_dsa_decode(num_requests=5, num_layers=2, steps=6, context=6000)
+    run_trace(w, w.steps, ctas_per_request=S, flags=NARROW)
+
+
+@pytest.mark.parametrize("policy", [hs.POLICY_LRU, hs.POLICY_FIFO, hs.POLICY_RANDOM])
+def test_narrow_blocks_shapes_groups_and_policies(policy):
+    # ragged k and B; B = 8192 (16 list entries per thread); groups with prefetch; page table not staged (shared lookups)
+    w = inputs.Workload("ragged", inputs.KIND_DSA_MIX, 3, 2, 1, 1000, 3001, 80, [5000, 7000, 2500], 6,
+                        keep=800, recent_window=300, seed=3, config_id=9)
+    run_trace(w, w.steps, flags=NARROW, policy=policy, policy_seed=3, pool_every=3)
+    w = inputs.Workload("wide", inputs.KIND_DSA_MIX, 2, 1, 1, 2048, 8192, 16, [30000, 20000], 4,
+                        keep=1500, recent_window=2048, seed=4, config_id=10)
+    run_trace(w, w.steps, flags=NARROW, policy=policy, policy_seed=3)
+    w = inputs.c3_dsa_long(0.5, steps=4, short_ctx=8192, long_ctx=65536, num_short=2)
+    run_trace(w, w.steps, use_prefetch=True, flags=NARROW, policy=policy, policy_seed=3)
+    w = inputs.c3_dsa_long(0.5, steps=3, short_ctx=90000, long_ctx=200000, num_short=2)
+    w.entry_bytes = 64
+    run_trace(w, w.steps, use_prefetch=True, ctas_per_request=2, flags=NARROW, policy=policy, policy_seed=3)
+
+
+def test_block_size_is_chosen_by_the_grid_and_refused_when_it_cannot_fit():
+    w = tiny_workload(2, 1, 1, 4, 8, 32, [20, 30])
+    pair = Pair(w)
+    assert pair.gpu.launch_geometry()["threads"] == 1024          # one wave: one block per SM
+    pair.close()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    w = tiny_workload(sms + 1, 1, 1, 4, 8, 32, [20] * (sms + 1), steps=4)
+    for flags, threads in ((0, 512), (hs.FLAG_WIDE_BLOCKS, 1024)):  # more blocks than SMs: two per SM unless told not to
+        pair = Pair(w, flags=flags | hs.FLAG_DEBUG_VALIDATE)
+        try:
+            assert pair.gpu.launch_geometry()["threads"] == threads
+            rng = np.random.default_rng(9)
+            for step in range(3):
+                pair.append()
+                rows = np.stack([inputs.random_rows(rng, 1, 4, pair.oracle.length(r), 0.1)[0] for r in range(sms + 1)])
+                pair.resolve_and_compare(0, rows)
+            pair.compare_state(0, requests=[0, sms])
+            pair.finish()
+        finally:
+            pair.close()
+    hist = [HostHistory(1, 40000, 16) for _ in range(2)]
+    try:
+        for flags in (hs.FLAG_NARROW_BLOCKS | hs.FLAG_WIDE_BLOCKS, hs.FLAG_NARROW_BLOCKS):
+            with pytest.raises(HiSparseError):                     # both at once; B beyond 16 list entries per thread
+                HiSparse(2, 1, 1, 8193 if flags == hs.FLAG_NARROW_BLOCKS else 64, 8, 16, [40000, 40000], [100, 100], hist,
+                         flags=flags)
+        with pytest.raises(HiSparseError):
+            HiSparse(2, 1, 1, 4096, 2049, 16, [40000, 40000], [5000, 5000], hist, flags=hs.FLAG_NARROW_BLOCKS)
+    finally:
+        for h in hist:
+            h.free()
+
+
 # ------------------------------------------------------------------ recency list left behind by hit-only resolves
 
 def _hit_only_rows(rng, pair, k, newest_too, layer=0):

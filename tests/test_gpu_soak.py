@@ -1,6 +1,7 @@
 """Randomised parity soak: seeded random geometries (B, k, N, layer groups, record sizes, context lengths on both
-sides of the page-table staging limit), cluster sizes, replacement policies, padding and repeated positions — every
-step compared bit for bit with the oracle (tables, counts, LRU state, plans, bytes)."""
+sides of the page-table staging limit), cluster sizes, block sizes, eager or lazy recency list, replacement policies,
+padding, repeated positions and repeated rows (resolves without misses) — every step compared bit for bit with the
+oracle (tables, counts, LRU state, plans, bytes)."""
 import numpy as np
 import pytest
 import torch
@@ -14,6 +15,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("seed", [0, 1, 2, 3])
 def test_random_configurations(seed):
     rng = np.random.default_rng(seed)
+    rng2 = np.random.default_rng(1000 + seed)     # geometry of the launch, repeated rows
     for _ in range(12):
         B = int(rng.choice([5, 33, 100, 257, 1000, 4096, 6000]))
         k = int(rng.integers(1, min(B, hs.MAX_TOP_K) + 1))
@@ -29,14 +31,28 @@ def test_random_configurations(seed):
         steps = 8
         w = inputs.Workload("soak", inputs.KIND_DSA_MIX, N, L, lpg, k, B, E, lens, steps, keep=int(k * rng.random()),
                             recent_window=int(rng.integers(1, 2000)), seed=int(rng.integers(1 << 30)), config_id=77)
-        pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE, ctas_per_request=S, policy=policy, policy_seed=5,
-                    oracle_bytes=E <= 1152)
+        flags = hs.FLAG_DEBUG_VALIDATE | (hs.FLAG_EAGER_ORDER if rng2.random() < 0.2 else 0)
+        narrow = rng2.random() < 0.5
+        try:
+            pair = Pair(w, flags=flags | (hs.FLAG_NARROW_BLOCKS if narrow else 0), ctas_per_request=S, policy=policy,
+                        policy_seed=5, oracle_bytes=E <= 1152)
+            assert pair.gpu.launch_geometry()["threads"] == (512 if narrow else 1024)
+        except hs.HiSparseError:                    # the shape does not allow 512-thread blocks
+            assert narrow
+            pair = Pair(w, flags=flags, ctas_per_request=S, policy=policy, policy_seed=5, oracle_bytes=E <= 1152)
+        hit_only_steps = rng2.random() < 0.5
+        prev = None
         tr = inputs.Trace(w)
         side = torch.cuda.Stream() if lpg > 1 and rng.random() < 0.7 else None
         repeat = rng.random() < 0.3
         try:
             for _step in range(steps):
-                sel, appended, _ = tr.step()
+                if hit_only_steps and prev is not None and rng2.random() < 0.4:
+                    sel, appended = prev, False     # the same rows again: nothing misses, the list is left behind
+                else:
+                    sel, appended, _ = tr.step()
+                    sel = [x.copy() for x in sel]
+                prev = sel
                 if appended:
                     pair.append()
                 for layer in range(L):
