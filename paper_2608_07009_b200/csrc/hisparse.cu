@@ -5,8 +5,10 @@
 //   pool      uint8  [L][N][B+1][E]   cache pools; slot B of each (r, l) is the reserved newest-record slot
 //   slot_pos  int32  [N][G][B]        position held by each slot, -1 = empty
 //   last_use  uint32 [N][G][B]        recency stamps: 2t+1 hit at resolve t, 2t fetched at resolve t, 0 unused
-//   order     uint16 [N][G][B]        slots from least to most recent; always equal to sorting the slots by
-//                                     (last_use, slot).  Kept so that victim choice is a prefix scan, not a sort
+//   order     uint16 [N][G][B]        slots from least to most recent: equal to sorting the slots by (last_use,
+//                                     slot) whenever order_t == t.  Kept so that victim choice is a prefix scan,
+//                                     not a sort; resolves without misses leave it behind (rebuild_order)
+//   order_t   uint32 [N][G]           resolve count the list is current for
 //   pos2slot  int16  ragged [N][G][capacity[r]]  the page table (Sec. 3.2), -1 = host-only
 //   plan_*    int32  [N][G][k]        miss plan of the last anchor resolve (Sec. 3.5)
 // All step-dependent scalars (resolve counters, number of appends, plan sizes) live in device memory so
@@ -20,8 +22,10 @@
 // ++ hits by slot).  As soon as (position, victim) pairs exist the missing records travel host -> shared memory
 // -> cache slot with cp.async.bulk in both directions (Phase 4); the plan is published to the other blocks of the
 // cluster, which take their share of the records, so the fetch parallelism does not depend on the number of
-// requests.  The launch carries the programmatic-dependent-launch attribute: everything before
-// griddepcontrol.wait depends on nothing an earlier kernel wrote.
+// requests.  A resolve in which nothing missed stops after the lookups: slot table, hit stamps, counters.
+// The launch carries the programmatic-dependent-launch attribute: everything before
+// griddepcontrol.wait depends on nothing an earlier kernel wrote.  Blocks have 1024 threads and an SM each;
+// grids of more blocks than SMs run the 512-thread instantiation, two blocks per SM.
 #include "hisparse.h"
 
 #include <cuda_runtime.h>
