@@ -370,6 +370,32 @@ def test_list_catches_up_after_hit_only_runs(policy, B, k, S):
         pair.close()
 
 
+@pytest.mark.parametrize("flags", [0, hs.FLAG_NARROW_BLOCKS])
+def test_list_catches_up_after_long_hit_only_runs(flags):
+    """70 and 300 skipped resolves: 7 and 9 stable splits when the list is rebuilt."""
+    rng = np.random.default_rng(3)
+    B, k = 37, 9
+    w = tiny_workload(2, 1, 1, k, B, 32, [150, 90], steps=8)
+    pair = Pair(w, flags=flags | hs.FLAG_DEBUG_VALIDATE)
+    try:
+        for run in (70, 300):
+            for _ in range(3):
+                rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0] for r in range(2)])
+                pair.resolve_and_compare(0, rows, check_bytes=False)
+                pair.compare_state(0)
+            for i in range(run):
+                pair.resolve_and_compare(0, _hit_only_rows(rng, pair, k, newest_too=False), check_bytes=False)
+            pair.compare_state(0)
+            assert pair.gpu.order_lag(0, 0) >= run
+        rows = np.stack([inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.0)[0] for r in range(2)])
+        pair.resolve_and_compare(0, rows)
+        pair.compare_state(0)
+        assert pair.gpu.order_lag(0, 0) == 0
+        pair.finish()
+    finally:
+        pair.close()
+
+
 def test_eager_list_flag_gives_the_same_results_and_never_lags():
     rng = np.random.default_rng(77)
     B, k = 300, 130
