@@ -240,7 +240,7 @@ def run_reference(args):
         "cpu_baseline": {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
-    print(json.dumps(line), flush=True)
+    print(json.dumps(line), file=_json_out, flush=True)
 
 
 def workload_config(w, args):
@@ -252,6 +252,9 @@ def workload_config(w, args):
 
 
 # ----------------------------------------------------------------------------- our arm
+
+
+_json_out = sys.stdout
 
 
 def all_hit_point(dev, hbm_peak):
@@ -618,11 +621,17 @@ def run_ours(args):
         line["shared_layer_resolve_us"] = {"median": float(np.median(res_us[:, sh])), "mean": float(res_us[:, sh].mean())}
         line["prefetch"] = use_prefetch
     line.update(extra)
-    print(json.dumps(line), flush=True)
+    print(json.dumps(line), file=_json_out, flush=True)
 
 
 def main():
     args = parse_args()
+    # stdout carries exactly one JSON line: whatever a library writes to file descriptor 1 (NCCL's version banner
+    # under torchrun, for one) goes to stderr instead
+    global _json_out
+    sys.stdout.flush()
+    _json_out = os.fdopen(os.dup(1), "w")
+    os.dup2(2, 1)
     if args.impl == "reference":
         run_reference(args)
     else:
