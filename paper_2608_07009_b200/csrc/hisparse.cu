@@ -150,40 +150,42 @@ struct TmaFetch {
   uint8_t *pbase;
   const int32_t *s_pos, *s_slot;
   uint32_t ring, bar;      // shared-memory addresses of this thread's ring slots and mbarrier
-  int64_t E, total;        // record bytes, number of pieces to move in this request
-  int chunk, ppr, depth, io_threads, part, nparts;
+  int64_t total;           // number of pieces to move in this request
+  int part, nparts;
   int batch;
   uint32_t parity;
   bool active;
+  // The pipeline's geometry (record bytes, piece size, pieces per record, ring slots per thread, issuing threads) is
+  // read from the kernel's DevState argument where it is used: constant-bank reads instead of live registers.
 
   __device__ __forceinline__ void init(const DevState &d, int r, int layer, int m, const int32_t *pos,
                                        const int32_t *slot, unsigned char *ring_base, unsigned long long *bars,
                                        int part_, int nparts_) {
     const int tid = threadIdx.x;
-    E = d.E; chunk = d.io_chunk; depth = d.io_depth; io_threads = d.io_threads;
-    ppr = d.io_ppr;
-    total = (int64_t)m * ppr;
+    total = (int64_t)m * d.io_ppr;
     part = part_; nparts = nparts_;
     s_pos = pos; s_slot = slot;
     hbase = d.host[r] + (int64_t)layer * d.cap[r] * d.E;
     pbase = d.pool + (int64_t)layer * d.layer_pool_bytes + (int64_t)r * (d.B + 1) * d.E;
-    ring = smem_u32(ring_base) + (uint32_t)tid * (uint32_t)(depth * chunk);
+    ring = smem_u32(ring_base) + (uint32_t)tid * (uint32_t)(d.io_depth * d.io_chunk);
     bar = smem_u32(bars + tid);
     batch = 0; parity = 0;
-    active = tid < io_threads && m > 0 && !(d.flags & HISPARSE_FLAG_SKIP_IO);
+    active = tid < d.io_threads && m > 0 && !(d.flags & HISPARSE_FLAG_SKIP_IO);
   }
 
   // piece number of this thread's q-th transfer
-  __device__ __forceinline__ int64_t piece_of(int q) const {
-    return ((int64_t)q * io_threads + threadIdx.x) * nparts + part;
+  __device__ __forceinline__ int64_t piece_of(const DevState &d, int q) const {
+    return ((int64_t)q * d.io_threads + threadIdx.x) * nparts + part;
   }
 
   // Issues the loads of the next batch; false when this thread has nothing left.
-  __device__ __forceinline__ bool issue() {
+  __device__ __forceinline__ bool issue(const DevState &d) {
     if (!active) return false;
+    const int depth = d.io_depth, chunk = d.io_chunk, ppr = d.io_ppr;
+    const int64_t E = d.E;
     uint32_t bytes_total = 0;
     for (int s = 0; s < depth; ++s) {
-      const int64_t c = piece_of(batch * depth + s);
+      const int64_t c = piece_of(d, batch * depth + s);
       if (c >= total) break;
       const int piece = ppr == 1 ? 0 : (int)(c % ppr);
       const int64_t rest = E - (int64_t)piece * chunk;
@@ -192,7 +194,7 @@ struct TmaFetch {
     if (bytes_total == 0) { active = false; return false; }
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes_total) : "memory");
     for (int s = 0; s < depth; ++s) {
-      const int64_t c = piece_of(batch * depth + s);
+      const int64_t c = piece_of(d, batch * depth + s);
       if (c >= total) break;
       const int64_t rec = ppr == 1 ? c : c / ppr;
       const int piece = (int)(c - rec * ppr);
@@ -206,7 +208,7 @@ struct TmaFetch {
   }
 
   // Waits for the batch issued last, stores it to the cache slots and frees the ring slots.
-  __device__ __forceinline__ void complete(uint32_t *status) {
+  __device__ __forceinline__ void complete(const DevState &d, uint32_t *status) {
     if (!mbar_wait_bounded(bar, parity)) {
       atomicOr(status, HISPARSE_STATUS_TIMEOUT);
       active = false;
@@ -214,8 +216,10 @@ struct TmaFetch {
     }
     parity ^= 1u;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    const int depth = d.io_depth, chunk = d.io_chunk, ppr = d.io_ppr;
+    const int64_t E = d.E;
     for (int s = 0; s < depth; ++s) {
-      const int64_t c = piece_of(batch * depth + s);
+      const int64_t c = piece_of(d, batch * depth + s);
       if (c >= total) break;
       const int64_t rec = ppr == 1 ? c : c / ppr;
       const int piece = (int)(c - rec * ppr);
@@ -230,11 +234,11 @@ struct TmaFetch {
     ++batch;
   }
 
-  __device__ __forceinline__ void drain(uint32_t *status) {
+  __device__ __forceinline__ void drain(const DevState &d, uint32_t *status) {
     bool pending = active;  // a batch is in flight whenever the thread is still active here
     while (pending) {
-      complete(status);
-      pending = issue();
+      complete(d, status);
+      pending = issue(d);
     }
     // complete() already waited until every store of this thread had read its ring slot (wait_group.read), which
     // is what shared memory needs before the block exits; the writes themselves are complete at grid end.
@@ -537,10 +541,10 @@ __device__ __forceinline__ void rebuild_order(const int B, const int W, const ui
   __syncthreads();
 }
 
-// Everything the first block of a cluster does before the fetch can start: Phases 1-3 of Sec. 3.4.
-// IPT = entries of the recency order per thread (B <= IPT * kThreads), KPT = row entries per thread (k <= KPT * kThreads).  On return s_plan_pos[i] / s_plan_slot[i] hold the position and
-// the victim slot of the i-th miss, s_out[j] the slot of every row entry (or -1 / a duplicate marker), s_order
-// the untouched slots compacted at its front, and s_hitbits / s_vicbits the per-slot marks.
+// Everything the first block of a cluster does before the fetch can start: Phases 1-2 of Sec. 3.4 and the list of
+// misses.  KPT = row entries per thread (k <= KPT * T).  On return s_plan_pos[i] holds the position of the i-th miss,
+// s_out[j] the slot of every row entry that hit (or -1, a duplicate marker, or the rank of its miss), s_hitbits the
+// hit marks and s_order the staged recency list; `fast` = nothing missed (and the list may be left behind).
 template <int T, int IPT, int KPT>
 __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r, const int64_t rg, const int32_t *row,
                                                  int32_t *s_sel, int32_t *s_out, int32_t *s_plan_pos,
@@ -550,7 +554,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
                                                  const int64_t p2s_off_r, unsigned long long *stamps,
                                                  unsigned char *s_ring, unsigned long long *s_bars,
                                                  const uint32_t t_now, int *s_warp_pre, int16_t *s_got, const int S,
-                                                 const uint32_t order_t, int &m, int &n_nonhit, uint32_t &my_status, bool &fast) {
+                                                 int &m, uint32_t &my_status, bool &fast) {
   const int tid = threadIdx.x;
   const int k = d.k, B = d.B, H = d.H;
   const uint32_t mask = (uint32_t)(H - 1);
@@ -675,7 +679,6 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     // is left as it is (rebuild_order brings it up to date in the next resolve that needs victims).
     fast = true;
     m = 0;
-    n_nonhit = 0;
     return;
   }
   if (timers && tid == 0) stamps[10] = clock64();
@@ -694,17 +697,50 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
     __syncthreads();
   }
   if (timers && tid == 0) stamps[11] = clock64();
+
+  // Phase 3, first half: the misses in selection order (one block scan; thread t owns KPT consecutive row entries).
+  // Their positions are all the fetch needs to start loading; the victims are only needed when a record is stored.
+  {
+    uint32_t miss_mask = 0;
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) {
+      const int j = tid * KPT + i;
+      if (j < k && s_out[j] == kMiss) miss_mask |= 1u << i;
+    }
+    int mrank = block_scan_excl(__popc(miss_mask), s_warp, m);
+#pragma unroll
+    for (int i = 0; i < KPT; ++i)
+      if ((miss_mask >> i) & 1u) {
+        const int j = tid * KPT + i;
+        s_plan_pos[mrank] = s_sel[j];      // position of the mrank-th miss
+        s_out[j] = kRankBase - mrank;      // its slot is the mrank-th victim, looked up when the table is written
+        ++mrank;
+      }
+  }
+  if (timers && tid == 0) stamps[12] = clock64();
+  __syncthreads();
+}
+
+// Phase 3, second half (runs while the first loads are in flight): brings the recency list up to date if it lags,
+// then ONE block scan over the non-hit slots in recency order.  Thread t owns IPT consecutive entries of the list.
+// On return s_plan_slot[i] holds the victim of the i-th miss, s_vicbits the victims' marks, s_order the untouched
+// slots compacted at its front and n_nonhit the number of slots without a hit.
+template <int T, int IPT>
+__device__ __forceinline__ void choose_victims(const DevState &d, const int r, const int64_t rg, const int m,
+                                               int32_t *s_plan_slot, unsigned long long *s_tab, const uint32_t *s_hitbits,
+                                               uint32_t *s_vicbits, uint16_t *s_order, int *s_warp, int *s_warp_pre,
+                                               unsigned long long *stamps, const uint32_t t_now, const uint32_t order_t,
+                                               int &n_nonhit) {
+  const int tid = threadIdx.x;
+  const int B = d.B;
+  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
   if (order_t != t_now - 1u) {
     const uint32_t *last_use = d.last_use + rg * B;
     rebuild_order<T, IPT>(B, d.W, last_use, 2u * order_t + 2u, t_now - 1u - order_t, s_order, s_vicbits, s_warp_pre, s_warp);
   }
-  if (timers && tid == 0) stamps[12] = clock64();
-
-  // Phase 3: ONE block scan over packed counts (non-hit slots in recency order | misses in selection order).
-  // Thread t owns IPT consecutive entries of the recency order and KPT consecutive row entries.
   {
     int slot[IPT];
-    uint32_t nh_mask = 0, miss_mask = 0;
+    uint32_t nh_mask = 0;
 #pragma unroll
     for (int i = 0; i < IPT; ++i) {
       const int q = tid * IPT + i;
@@ -714,24 +750,7 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
         if (!((s_hitbits[slot[i] >> 5] >> (slot[i] & 31)) & 1u)) nh_mask |= 1u << i;
       }
     }
-#pragma unroll
-    for (int i = 0; i < KPT; ++i) {
-      const int j = tid * KPT + i;
-      if (j < k && s_out[j] == kMiss) miss_mask |= 1u << i;
-    }
-    int total;
-    const int excl = block_scan_excl((__popc(nh_mask) << 16) | __popc(miss_mask), s_warp, total);
-    m = total & 0xffff;
-    n_nonhit = total >> 16;
-    int mrank = excl & 0xffff, nrank = excl >> 16;
-#pragma unroll
-    for (int i = 0; i < KPT; ++i)
-      if ((miss_mask >> i) & 1u) {
-        const int j = tid * KPT + i;
-        s_plan_pos[mrank] = s_sel[j];      // position of the mrank-th miss
-        s_out[j] = kRankBase - mrank;      // its slot is the mrank-th victim, looked up when the table is written
-        ++mrank;
-      }
+    int nrank = block_scan_excl(__popc(nh_mask), s_warp, n_nonhit);
     if (d.policy == HISPARSE_POLICY_LRU) {
       // the i-th miss (selection order) takes the i-th non-hit slot of the recency order
 #pragma unroll
@@ -886,7 +905,7 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
 #define HS_META(IPT, KPT)                                                                                         \
   resolve_metadata<T, IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
                              s_order, s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t,      \
-                             s_vicpre, s_got, S, order_t, m, n_nonhit, my_status, fast)
+                             s_vicpre, s_got, S, m, my_status, fast)
     if constexpr (T == kThreads) {
       if (k <= 2 * T) {
         if (B <= 4 * T) HS_META(4, 2);
@@ -942,9 +961,25 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
         if (timers) stamps[4] = global_ns();
       }
     } else {
-      // Phase 4 starts here: the first batch of host loads is in flight while the metadata is written back
+      // Phase 4 starts here, with the positions of the misses: the first batch of host loads is in flight while the
+      // victims are chosen (a record's slot is only needed when it is stored) and the metadata is written back
       fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
-      fetch.issue();
+      fetch.issue(d);
+#define HS_VICT(IPT)                                                                                              \
+  choose_victims<T, IPT>(d, r, rg, m, s_plan_slot, s_tab, s_hitbits, s_vicbits, s_order, s_warp, s_vicpre, stamps, t, \
+                         order_t, n_nonhit)
+      if constexpr (T == kThreads) {
+        if (B <= 4 * T) HS_VICT(4);
+        else if (B <= 8 * T) HS_VICT(8);
+        else HS_VICT(16);
+      } else {
+        if (B <= 8 * T) HS_VICT(8);
+        else HS_VICT(16);
+      }
+#undef HS_VICT
+      // same state as right after the first issue, recomputed instead of kept in registers across the victim choice
+      fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
+      fetch.active = fetch.active && fetch.piece_of(d, 0) < fetch.total;
       // Phase 5, metadata half: page table, slot array, stamps, plan
       int32_t *slot_pos = d.slot_pos + rg * B;
       uint32_t *last_use = d.last_use + rg * B;
@@ -1047,13 +1082,13 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       for (int i = tid; i < m; i += T) { s_plan_pos[i] = __ldcg(pp + i); s_plan_slot[i] = __ldcg(ps + i); }
       __syncthreads();
       fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, part, S);
-      fetch.issue();
+      fetch.issue(d);
     }
   }
   // Phase 4, rest: wait for the batches, store them into the cache slots, issue what is left.  Whatever follows
   // in the stream may be scheduled from here on (it still waits for this grid to finish before it reads).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  fetch.drain(d.status);
+  fetch.drain(d, d.status);
   if (timers) {
     __syncthreads();
     if (tid == 0) {
@@ -1082,8 +1117,8 @@ __global__ void __launch_bounds__(kThreads, 1) replay_kernel(const DevState d, c
   __syncthreads();
   TmaFetch fetch;
   fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, part, S);
-  fetch.issue();
-  fetch.drain(d.status);
+  fetch.issue(d);
+  fetch.drain(d, d.status);
 }
 
 // A shared layer reuses its anchor's slot table (same local slots, same request offsets) and counts.
