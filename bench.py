@@ -298,9 +298,9 @@ def all_hit_point(dev, hbm_peak):
     achieved = ALGO_BYTES_PER_HIT * N * k / t / 1e9
     return {"bound": "hbm", "achieved": achieved, "peak": hbm_peak["value"], "unit": "GB/s",
             "frac": achieved / hbm_peak["value"], "peak_source": hbm_peak["source"],
-            "traffic": 75137792 if N == 2048 else None,
+            "traffic": 76281344 if N == 2048 else None,
             "traffic_source": "profiles/resolve_kernel_all_hit_set_full.md",
-            "issue_bound_note": "ncu: 47 % of peak instruction issue, 16 % of DRAM throughput: issue/latency bound",
+            "issue_bound_note": "ncu: 47 % of peak instruction issue, 17 % of DRAM throughput: issue/latency bound",
             "workload": "scaled all-hit point: %d requests x 1 layer, k=%d, B=%d, every selection hits" % (N, k, B),
             "algorithmic_bytes_per_launch": ALGO_BYTES_PER_HIT * N * k, "launch_us": t * 1e6,
             "selections_per_s": N * k / t, "ctas_per_request": geo["ctas_per_request"]}
@@ -601,7 +601,7 @@ def run_ours(args):
             "frac": achieved / link_peak if link_peak else None,
             "peak_source": "measured in this run: best of 10 bulk pinned cudaMemcpyAsync H2D of 1 GiB",
             "kernel": "resolve_kernel",
-            "traffic": 2743296 if (w.name, N) == ("c2_dsa_decode", 32) else None,
+            "traffic": 2883328 if (w.name, N) == ("c2_dsa_decode", 32) else None,
             "traffic_source": "profiles/resolve_kernel_c2_set_full.md: dram__bytes_read + dram__bytes_write of one launch",
             "algorithmic_bytes_per_launch": algo_bytes_per_launch, "launch_us": avg_launch_s * 1e6,
             "launch_us_method": "CUDA events around each step's graph replay / resolve launches per step"},

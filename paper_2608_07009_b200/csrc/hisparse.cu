@@ -17,10 +17,11 @@
 // The Resolve kernel (Sec. 3.4, Phases 1-5) runs one thread-block cluster per request.  The cluster's first
 // block does the metadata: it stages the selected row, the recency order and (when it fits) the request's slice of
 // the page table in shared memory with bulk copies, looks every selection up in the page table, marks hit slots in
-// a bitset, compacts the misses in selection order and walks the recency order once (one block scan) to split the
-// non-hit slots into the first m (victims) and the rest, and rewrites the order as (untouched ++ victims by slot
-// ++ hits by slot).  As soon as (position, victim) pairs exist the missing records travel host -> shared memory
-// -> cache slot with cp.async.bulk in both directions (Phase 4); the plan is published to the other blocks of the
+// a bitset and compacts the misses in selection order (one block scan).  As soon as the missing positions exist the
+// records start travelling host -> shared memory -> cache slot with cp.async.bulk in both directions (Phase 4);
+// while the first loads fly the block walks the recency order once (a second scan) to split the non-hit slots
+// into the first m (victims, needed only when a record is stored) and the rest, and rewrites the order as
+// (untouched ++ victims by slot ++ hits by slot); the plan is published to the other blocks of the
 // cluster, which take their share of the records, so the fetch parallelism does not depend on the number of
 // requests.  A resolve in which nothing missed stops after the lookups: slot table, hit stamps, counters.
 // The launch carries the programmatic-dependent-launch attribute: everything before
