@@ -491,7 +491,7 @@ def run_ours(args):
                   "kernel_span": float((st[:, 6].max() - st[:, 0].min()) / 1e3),
                   "unit": "us, mean over requests, last anchor launch"}
         cyc = st[:, [15, 8, 9, 10, 11, 12, 13, 14]]
-        phases["cycles_issue_landed_lookup_count_barrier_scan_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
+        phases["cycles_issue_landed_lookup_dedup_missscan_victims_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
 
     total_s_max, sel_total = sharding.aggregate(total_s, sel_count, dev)
 
