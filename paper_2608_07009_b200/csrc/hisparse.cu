@@ -1000,12 +1000,10 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       if (tid == 0) d.plan_n[rg] = m;
     }
     if (my_status) atomicOr(d.status, my_status);
-    if (S > 1) {
-      __threadfence();
-      __syncthreads();
-    }
   }
-  // The plan is public: the other blocks of the cluster start fetching while this one publishes.
+  // The plan is public: the other blocks of the cluster start fetching while this one publishes.  Every thread
+  // arrives with release semantics after its own plan writes and every reader waits with acquire semantics, which
+  // orders them at cluster scope: no separate fence.
   if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
   if (part == 0 && !fast) {
