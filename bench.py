@@ -431,7 +431,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         cold_ms = e0.elapsed_time(e1)
         launches_per_step = {}
-        for kind in sorted({x is not None for x in kv_dev[1:]}):
+        for kind in sorted({x is not None for x in kvs[1:]}):      # the end-to-end steps included
             gph = torch.cuda.CUDAGraph()
             gph.capture_begin()
             launches_per_step[kind] = enqueue_step(kind, stream=main)
@@ -552,6 +552,27 @@ def run_ours(args):
                             "note": "graph of %d resolves on the last step's rows, no append, L2 flushed between replays"
                                     % L}
             del gph
+    # ---- the consumer's gather (stand-in for sparse attention reading the cache through the slot table) ----
+    consumer = None
+    if not args.skip_io and N * k * E <= (2 << 30):
+        with torch.cuda.stream(main):
+            out_buf = torch.empty((N, k, E), dtype=torch.uint8, device=dev)
+            ts = []
+            for i in range(3 + 8):
+                flush.zero_()
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(main)
+                gpu.gather(0, tabs[0], out_buf, stream=main)
+                b_.record(main)
+                b_.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b_) * 1e-3)
+            t_g = statistics.mean(ts)
+            peak = hbm_peak()
+            consumer = {"kernel": "gather_kernel", "launch_us": t_g * 1e6, "bytes_read_plus_written": 2 * N * k * E,
+                        "hbm_gb_s": 2 * N * k * E / t_g / 1e9, "frac_of_hbm_peak": 2 * N * k * E / t_g / 1e9 / peak["value"],
+                        "peak_source": peak["source"]}
+            del out_buf
     status |= gpu.status()
     del graphs
     gpu.close()
@@ -612,7 +633,7 @@ def run_ours(args):
         "misses_per_request_layer": float(miss_h[:, anchor_layers].mean()),
         "host_link": {"memcpy_peak_gb_s": link_peak, "sm_issued_read_gb_s": sm_read,
                       "note": "copy-only kernel, 148 blocks, random records of this workload's size"},
-        "cold_step_ms": cold_ms, "hit_only_step": hit_only, "status_bits": status, "launch_geometry": geo, "setup_s": setup_s,
+        "cold_step_ms": cold_ms, "hit_only_step": hit_only, "consumer_gather": consumer, "status_bits": status, "launch_geometry": geo, "setup_s": setup_s,
     }
     if phases:
         line["phases_us"] = phases

@@ -184,7 +184,7 @@ const void *hisparse_layer_pool(const hisparse_t *h, int layer);
 
 /* Stand-in for the sparse-attention consumer (Sec. 3.4 Phase 5: "the downstream gather can read
  * the selected records directly from the GPU cache"): copies the record of every table entry into
- * out_dev, uint8 [N][k][E]; entries with table value -1 are zero-filled. */
+ * out_dev, uint8 [N][k][E], 16-byte aligned (EINVAL otherwise); entries with table value -1 are zero-filled. */
 int hisparse_gather(hisparse_t *h, int layer, const int32_t *slot_table_dev, void *out_dev, void *stream);
 
 /* Exactness check of Sec. 3.1 ("HiSparse may change where entries reside, not the selected

@@ -1182,20 +1182,56 @@ __global__ void write_through_kernel(const DevState d) {
 // ------------------------------------------------------------------------------------------ consumer stand-ins
 
 // One warp per table entry: out[r][j] = pool[table[r][j]] (zeros for -1).
-__global__ void gather_kernel(const DevState d, const int layer, const int32_t *__restrict__ table,
-                              uint8_t *__restrict__ out) {
-  const int lane = threadIdx.x & 31;
-  const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+constexpr int kGatherThreads = 128;
+
+// Stand-in for the consumer's gather (Sec. 3.4 Phase 5): out[e] = pool[table[e]].  Copy-only, so it is written like
+// the fetch: every thread moves pieces of at most `chunk` bytes cache slot -> shared memory -> out with bulk copies
+// (one ring slot and one mbarrier per thread; the first `active` threads of a block take part, so that two blocks
+// fit an SM).  Entries with table value -1 are filled from a page of zeros.  Dynamic shared memory:
+// [kGatherThreads mbarriers][chunk bytes of zeros][active * chunk bytes of ring].
+__global__ void __launch_bounds__(kGatherThreads)
+gather_kernel(const DevState d, const int layer, const int32_t *__restrict__ table, uint8_t *__restrict__ out,
+              const int chunk, const int active) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem_raw);
+  unsigned char *zeros = smem_raw + kGatherThreads * 8;
+  unsigned char *ring = zeros + chunk;
+  const int tid = threadIdx.x;
+  for (int o = tid * 16; o < chunk; o += kGatherThreads * 16) *reinterpret_cast<uint4 *>(zeros + o) = make_uint4(0, 0, 0, 0);
+  if (tid < active) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + tid)) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the zeros are read by bulk stores
+  __syncthreads();
+  if (tid >= active) return;
   const uint8_t *pool = d.pool + (int64_t)layer * d.layer_pool_bytes;
-  for (int64_t e = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); e < (int64_t)d.N * d.k; e += nwarps) {
+  const int64_t E = d.E;
+  const int ppr = (int)((E + chunk - 1) / chunk);
+  const int64_t total = (int64_t)d.N * d.k * ppr, stride = (int64_t)gridDim.x * active;
+  const uint32_t slot = smem_u32(ring) + (uint32_t)tid * (uint32_t)chunk, bar = smem_u32(bars + tid);
+  uint32_t parity = 0;
+  for (int64_t c = (int64_t)blockIdx.x * active + tid; c < total; c += stride) {
+    const int64_t e = ppr == 1 ? c : c / ppr;
+    const int piece = (int)(c - e * ppr);
+    const int64_t rest = E - (int64_t)piece * chunk;
+    const uint32_t bytes = (uint32_t)(rest < chunk ? rest : chunk);
     const int32_t s = table[e];
-    uint4 *dst = reinterpret_cast<uint4 *>(out + e * d.E);
-    if (s < 0) {
-      for (uint32_t u = lane; u < d.upe; u += 32) dst[u] = make_uint4(0, 0, 0, 0);
-    } else {
-      const uint4 *src = reinterpret_cast<const uint4 *>(pool + (int64_t)s * d.E);
-      for (uint32_t u = lane; u < d.upe; u += 32) dst[u] = src[u];
+    uint8_t *dst = out + e * E + (int64_t)piece * chunk;
+    uint32_t from = smem_u32(zeros);
+    if (s >= 0) {
+      const uint8_t *src = pool + (int64_t)s * E + (int64_t)piece * chunk;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(slot), "l"(src), "r"(bytes), "r"(bar) : "memory");
+      if (!mbar_wait_bounded(bar, parity)) {
+        atomicOr(d.status, HISPARSE_STATUS_TIMEOUT);
+        return;
+      }
+      parity ^= 1u;
+      from = slot;
     }
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(from), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the ring slot may be overwritten
   }
 }
 
@@ -1318,6 +1354,7 @@ struct hisparse {
   DevState d{};
   int device = 0;
   int S = 1, T = kThreads;
+  int sm_count = 1;
   size_t resolve_smem = 0, replay_smem = 0;
   std::vector<int64_t> cap, init_len, p2s_off;
   int64_t p2s_total = 0;
@@ -1498,6 +1535,8 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
+  h->sm_count = sm_count;
+  if (cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
   // Block size.  One 1024-thread block per SM gives a request the whole SM and all of its shared memory for the
   // fetch ring.  When the grid takes several waves anyway (more blocks than SMs), two 512-thread blocks per SM hide
   // each other's dependent trips to memory; each then gets half of the SM's shared memory.
@@ -1769,7 +1808,12 @@ const void *hisparse_layer_pool(const hisparse_t *h, int layer) {
 
 int hisparse_gather(hisparse_t *h, int layer, const int32_t *slot_table_dev, void *out_dev, void *stream) {
   if (!h || layer < 0 || layer >= h->d.L || !slot_table_dev || !out_dev) return HISPARSE_EINVAL;
-  gather_kernel<<<592, 256, 0, as_stream(stream)>>>(h->d, layer, slot_table_dev, static_cast<uint8_t *>(out_dev));
+  if ((uintptr_t)out_dev & 15) return HISPARSE_EINVAL;  // bulk copies need 16-byte aligned addresses
+  const int chunk = (int)std::min<int64_t>(h->d.E, 8192);
+  const int active = (int)std::min<int64_t>(kGatherThreads, (96 * 1024) / chunk);
+  const size_t smem = (size_t)kGatherThreads * 8 + (size_t)chunk + (size_t)active * chunk;
+  gather_kernel<<<2 * h->sm_count, kGatherThreads, smem, as_stream(stream)>>>(h->d, layer, slot_table_dev,
+                                                                             static_cast<uint8_t *>(out_dev), chunk, active);
   HS_CUDA(cudaGetLastError());
   return HISPARSE_OK;
 }
