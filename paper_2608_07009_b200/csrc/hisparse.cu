@@ -73,6 +73,8 @@ struct DevState {
   uint16_t *order;
   int16_t *pos2slot;               // page table entries are slots (< 16384) or -1
   const int64_t *cap, *init_len, *p2s_off;
+  int64_t uni_cap, uni_init_len;   // capacity / initial length when every request has the same (else -1): the kernels
+                                   // then need no load for them and for p2s_off = r * G * capacity
   uint8_t *const *host;
   uint32_t *t;
   uint32_t *order_t;               // [N][G] resolve count up to which `order` is current; null = the list is never left stale
@@ -862,7 +864,9 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
     if (tid < 4) s_misc[tid] = 0;
   }
-  const int64_t cap_r = d.cap[r], init_len_r = d.init_len[r], p2s_off_r = d.p2s_off[r];  // fixed at create
+  const bool uni = d.uni_cap >= 0;  // fixed at create
+  const int64_t cap_r = uni ? d.uni_cap : d.cap[r], init_len_r = uni ? d.uni_init_len : d.init_len[r],
+                p2s_off_r = uni ? (int64_t)r * d.G * d.uni_cap : d.p2s_off[r];
   if (part == 0 && tid < 3) {
     // Warm L2 with what Phase 1 will stage (row, recency order, page-table slice).  A prefetch consumes nothing, and
     // L2 is where earlier kernels' writes land, so this is safe before the dependency wait; when the previous kernel
@@ -1530,6 +1534,10 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   int64_t off = 0;
   for (int r = 0; r < N; ++r) { h->p2s_off[r] = off; off += h->cap[r] * G; }
   h->p2s_total = off;
+  d.uni_cap = h->cap[0];
+  d.uni_init_len = h->init_len[0];
+  for (int r = 1; r < N; ++r)
+    if (h->cap[r] != h->cap[0] || h->init_len[r] != h->init_len[0]) d.uni_cap = d.uni_init_len = -1;
 
   int max_optin = 0, smem_per_sm = 0, sm_count = 0;
   if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
@@ -2128,6 +2136,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   lock.unlock();
 
   DevState d{};  // order_t stays null: the caller's recency list is brought up to date by every call
+  d.uni_cap = d.uni_init_len = -1;
   d.N = N; d.L = 1; d.lpg = 1; d.G = 1; d.B = B; d.k = k;
   d.H = hash_size(k); d.W = (B + 31) / 32;
   d.hshift = 32;
