@@ -1,5 +1,5 @@
-"""Builds the CUDA library in-tree: `nvcc` cross-compiles csrc/hisparse.cu for sm_100a into
-`_hisparse.so` next to this file (no GPU needed to build)."""
+"""Builds the CUDA library in-tree: `nvcc` cross-compiles csrc/hisparse.cu (which includes the other files of
+csrc/) for sm_100a into `_hisparse.so` next to this file (no GPU needed to build)."""
 from __future__ import annotations
 
 import os
@@ -19,7 +19,9 @@ def needs_build() -> bool:
     if not os.path.exists(SO):
         return True
     t = os.path.getmtime(SO)
-    return any(os.path.getmtime(p) > t for p in (SRC, HEADER))
+    csrc = os.path.dirname(SRC)          # hisparse.cu includes the other files of csrc/: one translation unit
+    deps = [os.path.join(csrc, f) for f in os.listdir(csrc)] + [HEADER]
+    return any(os.path.getmtime(p) > t for p in deps)
 
 
 def build_cuda(force: bool = False, verbose: bool = False) -> str:
