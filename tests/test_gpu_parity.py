@@ -340,7 +340,7 @@ def _hit_only_rows(rng, pair, k, newest_too, layer=0):
 
 
 @pytest.mark.parametrize("policy", [hs.POLICY_LRU, hs.POLICY_FIFO, hs.POLICY_RANDOM])
-@pytest.mark.parametrize("B,k,S", [(4, 2, 1), (12, 5, 2), (40, 17, 1), (300, 130, 4), (5000, 2100, 1)])
+@pytest.mark.parametrize("B,k,S", [(4, 2, 1), (12, 5, 2), (40, 17, 1), (300, 130, 4), (5000, 2100, 1), (16384, 257, 2)])
 def test_list_catches_up_after_hit_only_runs(policy, B, k, S):
     """Runs of 1..9 resolves in which nothing misses (the list is left behind and only stamps are written), each
     followed by resolves with misses (the list is re-sorted before victims are taken): everything still equals the
