@@ -107,7 +107,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -420,6 +420,10 @@ def run_ours(args):
     # one CUDA graph per kind of step, captured from the public API calls.
     graphs = {}
     torch.cuda.synchronize()
+    # clocks and throttle reasons are sampled from the cold step to the end of the timed region (the region alone
+    # lasts a few tens of milliseconds, about one sample)
+    sampler = ClockSampler(local)
+    sampler.start()
     with torch.cuda.stream(main):
         # cold step (everything misses), eager
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -447,8 +451,6 @@ def run_ours(args):
         barrier()
 
         # ---- timed region: K graph replays, inputs resident in HBM, L2 flushed between steps ----
-        sampler = ClockSampler(local)
-        sampler.start()
         step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         launches = 0
         for s_ in range(K):
