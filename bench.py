@@ -620,7 +620,9 @@ def run_ours(args):
         "gpu_launches": launches,
         "clocks": clocks,
         "roofline": {
-            "bound": "host_link", "achieved": achieved, "peak": link_peak, "unit": "GB/s",
+            "bound": "host_link", "bound_note": "the fetch over the host link (PCIe Gen5 x16) bounds a miss-heavy resolve, "
+            "neither HBM nor the tensor cores; the all-hit path is reported against HBM in roofline_all_hit",
+            "achieved": achieved, "peak": link_peak, "unit": "GB/s",
             "frac": achieved / link_peak if link_peak else None,
             "peak_source": "measured in this run: best of 10 bulk pinned cudaMemcpyAsync H2D of 1 GiB",
             "kernel": "resolve_kernel",
