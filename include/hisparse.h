@@ -125,7 +125,7 @@ int hisparse_create(const hisparse_config_t *cfg, hisparse_t **out);
 int hisparse_destroy(hisparse_t *h);
 
 /* Sec. 3.3 step (4) "Write-through of generated KV": every request appends one record per layer.
- * new_kv_dev is device memory [N][L][E]; request r's records land at position len[r], which then
+ * new_kv_dev is device memory [N][L][E], 16-byte aligned (EINVAL otherwise); request r's records land at position len[r], which then
  * grows by one.  The records are placed in the reserved slot of each (request, layer) cache, so
  * the newest position is always resident, and written through to the host history on the
  * library's backup stream (on `stream` itself with INLINE_WRITE_THROUGH), ordered by events so
@@ -182,13 +182,13 @@ int hisparse_join(hisparse_t *h, void *stream);
  * gathers from with the slot table).  Valid until destroy. */
 const void *hisparse_layer_pool(const hisparse_t *h, int layer);
 
-/* Stand-in for the sparse-attention consumer (Sec. 3.4 Phase 5: "the downstream gather can read
- * the selected records directly from the GPU cache"): copies the record of every table entry into
+/* Stand-in for the sparse-attention consumer, which takes the selected records out of the GPU cache through
+ * the slot table (Sec. 3.4 Phase 5): copies the record of every table entry into
  * out_dev, uint8 [N][k][E], 16-byte aligned (EINVAL otherwise); entries with table value -1 are zero-filled. */
 int hisparse_gather(hisparse_t *h, int layer, const int32_t *slot_table_dev, void *out_dev, void *stream);
 
-/* Exactness check of Sec. 3.1 ("HiSparse may change where entries reside, not the selected
- * positions or the outputs"): for every valid selection compares the E bytes its table entry
+/* Exactness check of Sec. 3.1 (the hierarchy moves records between tiers but never changes which positions are
+ * selected or what the attention computes from them): for every valid selection compares the E bytes its table entry
  * addresses with the host history's record at that position and adds the number of differing
  * selections to *mismatches_dev (int32, not cleared).  Joins the write-through first. */
 int hisparse_gather_check(hisparse_t *h, int layer, const int32_t *sel_dev, const int32_t *slot_table_dev,
@@ -284,8 +284,12 @@ int hisparse_scatter_read_probe(int device, const void *host_buf, size_t host_by
  * (HISPARSE_EINVAL).  One layer per state struct, no shared-selection groups, no prefetch.
  *
  * The first call on a device looks up the device address of the scratch array and raises the kernel's
- * shared-memory limit (with that device current); make that first call before any stream capture begins.
+ * shared-memory limit; make that first call before any stream capture begins.
  * Later calls only enqueue a memset of the scratch counters and the kernel on `stream`.
+ * Every call makes state->device the current device for its own duration and restores the caller's current
+ * device before it returns, so it may be called from a thread whose current device is another GPU.
+ * pool_dev and every address in host_layer_dev must be 16-byte aligned (the records travel as bulk copies);
+ * a misaligned pool_dev is refused with HISPARSE_EINVAL, the addresses in device memory cannot be checked.
  * Every call on a device shares the one scratch array, which keeps the previous call's contents: the call
  * clears what has to start from zero itself, and two calls whose kernels overlap on the GPU (different streams)
  * race on it — serialise them.

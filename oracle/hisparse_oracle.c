@@ -35,7 +35,9 @@
  *
  * Pins (tests/test_oracle_*.py): the worked example in tests/golden/, an independent ordered-list
  * LRU simulator on tiny random inputs, textbook LRU for k = 1, the B = k "keep only the current
- * top-k" closed form, byte identity with the host history, inverse maps, stamp ordering.
+ * top-k" closed form, byte identity with the host history, inverse maps, stamp ordering; for the
+ * RANDOM policy's key, the published first outputs of splitmix64 for seed 0 and a key worked out
+ * step by step in tests/golden/random_key_worked.txt.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -179,6 +181,11 @@ static uint32_t random_key(uint64_t seed, int r, int g, uint32_t t, int slot) {
   uint64_t a = oracle_mix64(seed ^ (((uint64_t)(uint32_t)r << 32) | (uint32_t)g));
   return (uint32_t)oracle_mix64(a + (((uint64_t)t << 32) | (uint32_t)slot));
 }
+
+/* Accessors for the pins of the two functions above (tests/test_oracle_policies.py): mix64 is the output function
+ * of the published splitmix64 generator, whose first outputs for seed 0 are known. */
+uint64_t oracle_mix64_value(uint64_t z) { return oracle_mix64(z); }
+uint32_t oracle_random_key_value(uint64_t seed, int r, int g, uint32_t t, int slot) { return random_key(seed, r, g, t, slot); }
 
 typedef struct { uint32_t stamp; int32_t slot; } cand_t;
 static int cmp_slot(const void *a, const void *b) {

@@ -67,6 +67,10 @@ def _L() -> ctypes.CDLL:
         L.oracle_clear_status.restype = None
         L.oracle_set_policy.argtypes = [vp, i32, ctypes.c_uint64]
         L.oracle_set_policy.restype = i32
+        L.oracle_mix64_value.argtypes = [ctypes.c_uint64]
+        L.oracle_mix64_value.restype = ctypes.c_uint64
+        L.oracle_random_key_value.argtypes = [ctypes.c_uint64, i32, i32, u32, i32]
+        L.oracle_random_key_value.restype = u32
         L.oracle_kv_footprint_bytes.argtypes = [i64, i64, i64, i64]
         L.oracle_kv_footprint_bytes.restype = i64
         _lib = L
@@ -75,6 +79,16 @@ def _L() -> ctypes.CDLL:
 
 def kv_footprint_bytes(N: int, L: int, slots: int, record_bytes: int) -> int:
     return int(_L().oracle_kv_footprint_bytes(N, L, slots, record_bytes))
+
+
+def mix64(z: int) -> int:
+    """The oracle's 64-bit mixing function (exported so that a test can pin it)."""
+    return int(_L().oracle_mix64_value(z & 0xFFFFFFFFFFFFFFFF))
+
+
+def random_key(seed: int, r: int, g: int, t: int, slot: int) -> int:
+    """The oracle's key of the RANDOM replacement policy for one slot."""
+    return int(_L().oracle_random_key_value(seed & 0xFFFFFFFFFFFFFFFF, r, g, t, slot))
 
 
 def _view(ptr: int, n: int, dtype) -> np.ndarray:

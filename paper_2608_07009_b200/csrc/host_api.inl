@@ -357,6 +357,7 @@ int hisparse_join(hisparse_t *h, void *stream) {
 
 int hisparse_append(hisparse_t *h, const void *new_kv_dev, void *stream) {
   if (!h || !new_kv_dev) return HISPARSE_EINVAL;
+  if ((uintptr_t)new_kv_dev & 15) return HISPARSE_EINVAL;  // the records are read as 16-byte vectors
   cudaStream_t st = as_stream(stream);
   const bool inline_wt = h->d.flags & HISPARSE_FLAG_INLINE_WRITE_THROUGH;
   if (h->wt_pending) {  // the previous write-through still reads the reserved slots

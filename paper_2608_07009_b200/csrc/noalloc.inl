@@ -33,12 +33,26 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
     return HISPARSE_EINVAL;
   if (N > HISPARSE_NOALLOC_MAX_REQUESTS || (int64_t)N * k > HISPARSE_NOALLOC_MAX_SELECTIONS) return HISPARSE_ETOOBIG;
 
+  // bulk copies write the fetched records straight into the pool: its base must be 16-byte aligned, like the
+  // histories (whose addresses live in device memory and cannot be checked here)
+  if ((uintptr_t)st->pool_dev & 15) return HISPARSE_EINVAL;
+
+  // Every call runs with the state's device current and leaves the caller's current device as it found it.
   const int dev = st->device;
+  int caller_dev = -1;
+  HS_CUDA(cudaGetDevice(&caller_dev));
+  struct DeviceGuard {
+    int restore;
+    ~DeviceGuard() { if (restore >= 0) cudaSetDevice(restore); }
+  } guard{-1};
+  if (caller_dev != dev) {
+    HS_CUDA(cudaSetDevice(dev));
+    guard.restore = caller_dev;
+  }
   std::unique_lock<std::mutex> lock(g_noalloc_mutex);
   if (!g_noalloc_ptr[dev]) {
     // Set-up, once per device, with that device current.  In host code the array's name is only a stand-in for
     // the symbol; the address a kernel can use comes from cudaGetSymbolAddress.
-    HS_CUDA(cudaSetDevice(dev));
     void *p = nullptr;
     HS_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
     int optin = 0;

@@ -5,7 +5,10 @@ import collections
 import numpy as np
 import pytest
 
+import os
+
 from oracle import Oracle, FLAG_NO_BYTES, POLICY_FIFO, POLICY_LRU, POLICY_RANDOM
+from oracle import oracle as oracle_mod
 from paper_2608_07009_b200 import inputs
 from lru_list_sim import ListLRUSim
 
@@ -15,6 +18,34 @@ POLICIES = {"lru": POLICY_LRU, "fifo": POLICY_FIFO, "random": POLICY_RANDOM}
 def make(B, k, length, policy, seed=0):
     return Oracle(1, 1, 1, B, k, 16, [length + 64], [length], None, FLAG_NO_BYTES, policy=POLICIES[policy],
                   policy_seed=seed)
+
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+GAMMA = 0x9E3779B97F4A7C15      # splitmix64's increment
+M64 = (1 << 64) - 1
+
+
+def test_mix64_is_the_published_splitmix64_output_function():
+    """splitmix64 seeded with 0 returns mix(0 + gamma), mix(0 + 2 gamma), ...; the oracle's mix64 adds gamma itself, so
+    mix64(0), mix64(gamma), mix64(2 gamma) must be the generator's published first three outputs for seed 0."""
+    published = [0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F]
+    assert [oracle_mod.mix64((i * GAMMA) & M64) for i in range(3)] == published
+
+
+def test_random_key_worked_example_and_argument_placement():
+    with open(os.path.join(GOLDEN, "random_key_worked.txt")) as f:
+        rows = [ln for ln in f if ln.strip() and not ln.startswith("#")]
+    vals = {ln.split("=")[0].strip(): int(ln.rsplit("=", 1)[1], 16) for ln in rows}
+    assert oracle_mod.mix64(vals["a0"]) == vals["a6"] and oracle_mod.mix64(vals["b0"]) == vals["b6"]
+    assert oracle_mod.random_key(0x1234, 3, 2, 5, 7) == vals["key"] == 0xC66719FE
+    # where each argument enters: request and group are folded into the seed word (high / low half), the resolve
+    # count and the slot are added to the mixed seed (high / low half); the key is the LOW half of the last mix
+    seed = 0x0123456789ABCDEF
+    key = oracle_mod.random_key
+    assert key(seed, 5, 9, 11, 13) == key(seed ^ (5 << 32) ^ 9, 0, 0, 11, 13)
+    base = oracle_mod.mix64(seed ^ (5 << 32 | 9))
+    assert key(seed, 5, 9, 11, 13) == oracle_mod.mix64((base + (11 << 32) + 13) & M64) & 0xFFFFFFFF
+    assert len({key(seed, r, g, t, s) for r in range(3) for g in range(3) for t in range(3) for s in range(3)}) == 81
 
 
 @pytest.mark.parametrize("policy", ["fifo", "random"])
