@@ -11,7 +11,7 @@ __global__ void __launch_bounds__(kThreads, 1) replay_kernel(const DevState d, c
   int32_t *s_plan_pos = reinterpret_cast<int32_t *>(smem_raw);
   int32_t *s_plan_slot = s_plan_pos + d.k;
   unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
-  unsigned char *s_ring = smem_raw + d.meta_smem + kBarBytes;
+  unsigned char *s_ring = smem_raw + d.meta_smem + d.bar_bytes;
   const int r = blockIdx.x / S, part = blockIdx.x - r * S;
   const int64_t rg = (int64_t)r * d.G + layer / d.lpg;
   const int m = d.plan_n[rg];
@@ -176,7 +176,7 @@ __global__ void validate_kernel(const DevState d, const int g) {
   const int32_t *slot_pos = d.slot_pos + rg * B;
   const uint32_t *last_use = d.last_use + rg * B;
   const uint16_t *order = d.order + rg * B;
-  const int16_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * d.cap[r];
+  const int16_t *p2s = d.pos2slot + d.p2s_off[r] + (int64_t)g * p2s_stride(d.cap[r]);
   for (int i = threadIdx.x; i < d.W; i += blockDim.x) seen[i] = 0u;
   __syncthreads();
   // a list that lags behind the stamps (resolves without misses) is still a permutation, but not sorted by them

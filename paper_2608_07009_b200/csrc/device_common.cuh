@@ -18,10 +18,8 @@ thread_local int g_last_cuda_error = 0;
 constexpr int kThreads = 1024;       // most threads per block of the resolve / replay kernels (one block per SM)
 constexpr int kThreadsSmall = 512;   // block size when the grid takes several waves: two blocks share an SM
 constexpr int kFetchUnroll = 4;      // 16-byte host loads in flight per thread (probe kernel)
-constexpr int kBarBytes = (kThreads + 2) * 8;  // one mbarrier per thread for the fetch ring + one for staging
-constexpr int32_t kMiss = -2;        // s_out marker: valid selection, not (yet) found resident
-constexpr int32_t kDupBase = -3;     // s_out marker: duplicate of row entry -(v + 3)
-constexpr int32_t kRankBase = -(1 << 20);  // s_out marker: the (kRankBase - v)-th miss of the row (slot = plan_slot of it)
+constexpr int32_t kMiss = -2;        // classification of a row entry: valid selection, not found resident
+constexpr int32_t kDupBase = -3;     // slot-table marker (kernel-internal): repeats the missing position of row entry -(v + 3)
 
 // Everything a kernel needs, passed by value.
 struct DevState {
@@ -34,7 +32,8 @@ struct DevState {
   int32_t *slot_pos;
   uint32_t *last_use;
   uint16_t *order;
-  int16_t *pos2slot;               // page table entries are slots (< 16384) or -1
+  int16_t *pos2slot;               // page table entries are slots (< 16384) or -1; request r's G slices start at
+                                   // p2s_off[r], p2s_stride(cap[r]) entries apart
   const int64_t *cap, *init_len, *p2s_off;
   int64_t uni_cap, uni_init_len;   // capacity / initial length when every request has the same (else -1): the kernels
                                    // then need no load for them and for p2s_off = r * G * capacity
@@ -46,7 +45,21 @@ struct DevState {
   int32_t *n_appends;
   uint32_t *ticket;
   uint32_t *status;
-  int meta_smem;                   // bytes of shared memory the metadata arrays take (ring follows)
+  // Dynamic shared memory of the resolve / replay kernels (byte offsets, fixed at create): the selected row at 0
+  // (its space is reused for the recency list once the row has been consumed), then the arrays below, the
+  // mbarriers at meta_smem and the staging ring of the fetch pipeline behind them.
+  int sm_plan_pos, sm_plan_slot;   // int32 [k] each: positions / victim slots of the misses, in selection order
+  int sm_missj;                    // uint16 [k]: row index of each miss
+  int sm_marks;                    // uint8: per-slot hit marks (a tag per request), zero-padded to a multiple of 2048
+  int marks_spare;                 // offset (from sm_marks) of a spare byte behind the padding
+  int sm_bits;                     // uint32 [4][W]: hit marks as a bitset, victim marks and their word-level prefix counts
+  int sm_hist;                     // int32 [260]: histogram of the RANDOM policy's radix select
+  int sm_got;                      // int16 [k]: page-table answers from the whole cluster (0 = not allocated)
+  int sm_misc;                     // int32 [64]: scratch of the block scans, per-request flags
+  int sm_tab;                      // uint64 [H]: table of the missing positions; -1 = it lives at the start of the ring
+                                   // and is cleared only once a miss has been seen
+  int meta_smem;                   // bytes of shared memory the arrays above take
+  int bar_bytes;                   // (threads + 2) mbarriers: one per thread for the fetch ring, two for staging
   int io_threads, io_depth, io_chunk;  // fetch pipeline: issuing threads, ring slots per thread, bytes per piece
   int ring_bytes;                  // io_threads * io_depth * io_chunk
   int io_ppr;                      // pieces per record = ceil(E / io_chunk)
@@ -64,6 +77,11 @@ __device__ __forceinline__ uint4 ld_host16(const void *p) {
                : "l"(p));
   return v;
 }
+
+// Entries between the page-table slices of consecutive groups of one request: the capacity rounded up to whole
+// 16-byte units, so that every slice of a library-owned table starts on a 16-byte boundary and can travel to shared
+// memory as one bulk copy (the padding entries stay -1).
+__host__ __device__ __forceinline__ int64_t p2s_stride(int64_t cap) { return (cap + 7) & ~(int64_t)7; }
 
 // Multiplicative hash of a position into a table of H = 2^(32 - shift) entries.
 __device__ __forceinline__ uint32_t hash_pos(int32_t p, int shift) {
@@ -100,6 +118,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   uint32_t done = 0;
   uint64_t t0 = 0;
   for (uint32_t spin = 0;; ++spin) {
+    // (no suspend-time hint: with a hint of 1 us a waiting warp was measured to sleep on, long after the phase had
+    // completed, which made the wait for 24 KB of staged inputs take 5 us)
     asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                  : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
@@ -126,7 +146,7 @@ struct TmaFetch {
 
   __device__ __forceinline__ void init(const DevState &d, int r, int layer, int m, const int32_t *pos,
                                        const int32_t *slot, unsigned char *ring_base, unsigned long long *bars,
-                                       int part_, int nparts_) {
+                                       int part_, int nparts_, uint32_t parity_ = 0) {
     const int tid = threadIdx.x;
     total = (int64_t)m * d.io_ppr;
     part = part_; nparts = nparts_;
@@ -135,7 +155,7 @@ struct TmaFetch {
     pbase = d.pool + (int64_t)layer * d.layer_pool_bytes + (int64_t)r * (d.B + 1) * d.E;
     ring = smem_u32(ring_base) + (uint32_t)tid * (uint32_t)(d.io_depth * d.io_chunk);
     bar = smem_u32(bars + tid);
-    batch = 0; parity = 0;
+    batch = 0; parity = parity_;  // the phase this thread's barrier is in (a block that loops over requests carries it along)
     active = tid < d.io_threads && m > 0 && !(d.flags & HISPARSE_FLAG_SKIP_IO);
   }
 
@@ -173,12 +193,16 @@ struct TmaFetch {
     return true;
   }
 
-  // Waits for the batch issued last, stores it to the cache slots and frees the ring slots.
-  __device__ __forceinline__ void complete(const DevState &d, uint32_t *status) {
+  // Waits for the batch issued last, stores it to the cache slots and frees the ring slots.  False = the bounded
+  // wait expired.
+  __device__ __forceinline__ bool complete(const DevState &d, uint32_t *status) {
     if (!mbar_wait_bounded(bar, parity)) {
+      // Give the loads in flight one more bounded chance to land before this thread stops using its ring slots: the
+      // block must not hand its shared memory to the next block while bulk copies are still writing into it.
       atomicOr(status, HISPARSE_STATUS_TIMEOUT);
+      mbar_wait_bounded(bar, parity);
       active = false;
-      return;
+      return false;
     }
     parity ^= 1u;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -198,24 +222,31 @@ struct TmaFetch {
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // ring slots reusable
     ++batch;
+    return true;
   }
 
-  __device__ __forceinline__ void drain(const DevState &d, uint32_t *status) {
+  // Returns false when a bounded wait expired (the barrier's phase is then unknown).
+  __device__ __forceinline__ bool drain(const DevState &d, uint32_t *status) {
     bool pending = active;  // a batch is in flight whenever the thread is still active here
+    bool ok = true;
     while (pending) {
-      complete(d, status);
+      ok = complete(d, status) && ok;
       pending = issue(d);
     }
     // complete() already waited until every store of this thread had read its ring slot (wait_group.read), which
     // is what shared memory needs before the block exits; the writes themselves are complete at grid end.
+    return ok;
   }
 };
 
+// Barriers [0, blockDim.x): one per thread of the fetch pipeline; the two behind them complete the staging of the
+// selected row + page-table slice and of the recency list.  Every thread of the block must pass a block barrier
+// after this call before any of the barriers is used.
 __device__ __forceinline__ void fetch_barriers_init(unsigned long long *bars, int io_threads) {
   if ((int)threadIdx.x < io_threads)
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + threadIdx.x)) : "memory");
-  if (threadIdx.x == 0)  // the staging barrier of the page-table slice
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + kThreads)) : "memory");
+  if (threadIdx.x < 2)
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + blockDim.x + threadIdx.x)) : "memory");
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 

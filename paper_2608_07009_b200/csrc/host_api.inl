@@ -5,7 +5,8 @@
 struct hisparse {
   DevState d{};
   int device = 0;
-  int S = 1, T = kThreads;
+  int S = 1, T = kThreads, minb = 1;   // blocks per request, threads per block, blocks of that size per SM
+  int clusters = 1;                    // clusters in a resolve launch: N, or one resident wave that loops over the requests
   int sm_count = 1;
   size_t resolve_smem = 0, replay_smem = 0;
   std::vector<int64_t> cap, init_len, p2s_off;
@@ -66,22 +67,59 @@ int hash_size(int k) {
   return H;
 }
 
-size_t resolve_smem_bytes(int B, int k) {
-  const int H = hash_size(k), W = (B + 31) / 32;
-  return (size_t)H * 8 + (size_t)4 * k * 4 + (size_t)4 * W * 4 + (size_t)((B + 7) & ~7) * 2 + (size_t)k * 2;
+// Lays out the dynamic shared memory of the resolve / replay kernels for blocks of `threads` threads.  `coop` =
+// the blocks of a cluster may share the page-table lookups (needs the answers array); `tab_in_ring` = the table of
+// missing positions shares the ring's memory instead of having its own.
+void layout_smem(DevState &d, int threads, bool coop, bool tab_in_ring) {
+  auto pad = [](size_t x) { return (x + 15) & ~(size_t)15; };
+  const size_t k = (size_t)d.k, B = (size_t)d.B, wpad = ((size_t)d.W + 3) & ~(size_t)3;
+  size_t o = std::max(pad(k * 4), pad(B * 2));   // the row, later the recency list
+  d.sm_plan_pos = (int)o;  o += pad(k * 4);
+  d.sm_plan_slot = (int)o; o += pad(k * 4);
+  d.sm_missj = (int)o;     o += pad(k * 2);
+  d.sm_marks = (int)o;     d.marks_spare = (int)((B + 2047) & ~(size_t)2047); o += (size_t)d.marks_spare + 16;
+  d.sm_bits = (int)o;      o += 4 * wpad * 4;   // hit and victim bitsets, two prefix arrays
+  d.sm_hist = (int)o;      o += 1040;
+  d.sm_misc = (int)o;      o += 256;
+  d.sm_got = coop ? (int)o : 0; o += coop ? pad(k * 2) : 0;
+  d.sm_tab = tab_in_ring ? -1 : (int)o; o += tab_in_ring ? 0 : (size_t)d.H * 8;
+  d.meta_smem = (int)((o + 127) & ~(size_t)127);
+  d.bar_bytes = (threads + 2) * 8;
+}
+
+// Geometry of the fetch pipeline for `ring_room` bytes of staging ring.  False when not even one piece fits (or, with
+// the table inside the ring, when the ring cannot hold it).
+bool layout_ring(DevState &d, int threads, int64_t ring_room) {
+  if (ring_room < 16) return false;
+  d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
+  const int slots = (int)(ring_room / d.io_chunk);
+  d.io_threads = std::min(slots, threads);
+  d.io_depth = std::min(slots / d.io_threads, 8);
+  d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
+  d.io_ppr = (int)((d.E + d.io_chunk - 1) / d.io_chunk);
+  if (d.sm_tab < 0 && (int64_t)d.H * 8 > ring_room) return false;
+  return true;
+}
+
+size_t kernel_smem_bytes(const DevState &d) {
+  // with the table inside the ring, the allocation covers the larger of the two
+  const size_t ring = d.sm_tab < 0 ? std::max<size_t>((size_t)d.ring_bytes, (size_t)d.H * 8) : (size_t)d.ring_bytes;
+  return (size_t)d.meta_smem + (size_t)d.bar_bytes + ring;
 }
 
 cudaStream_t as_stream(void *s) { return static_cast<cudaStream_t>(s); }
 
-const void *resolve_kernel_of(int threads) {
-  return threads == kThreadsSmall ? reinterpret_cast<const void *>(&resolve_kernel<kThreadsSmall>)
-                                  : reinterpret_cast<const void *>(&resolve_kernel<kThreads>);
+const void *resolve_kernel_of(int threads, int minb) {
+  if (threads == kThreadsSmall)
+    return minb >= 3 ? reinterpret_cast<const void *>(&resolve_kernel<kThreadsSmall, 3, true>)
+                     : reinterpret_cast<const void *>(&resolve_kernel<kThreadsSmall, 2, true>);
+  return reinterpret_cast<const void *>(&resolve_kernel<kThreads, 1, false>);
 }
 
 int launch_resolve(hisparse *h, int layer, const int32_t *sel, int32_t *table, int32_t *hits, int32_t *misses,
                    cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(h->d.N * h->S));
+  cfg.gridDim = dim3((unsigned)(h->clusters * h->S));
   cfg.blockDim = dim3((unsigned)h->T);
   cfg.dynamicSmemBytes = h->resolve_smem;
   cfg.stream = st;
@@ -94,10 +132,12 @@ int launch_resolve(hisparse *h, int layer, const int32_t *sel, int32_t *table, i
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (h->d.flags & HISPARSE_FLAG_NO_PDL) ? 1 : 2;
-  if (h->T == kThreadsSmall)
-    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreadsSmall>, h->d, layer, sel, table, hits, misses, h->S));
+  if (h->T == kThreadsSmall && h->minb >= 3)
+    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreadsSmall, 3, true>, h->d, layer, sel, table, hits, misses, h->S));
+  else if (h->T == kThreadsSmall)
+    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreadsSmall, 2, true>, h->d, layer, sel, table, hits, misses, h->S));
   else
-    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreads>, h->d, layer, sel, table, hits, misses, h->S));
+    HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreads, 1, false>, h->d, layer, sel, table, hits, misses, h->S));
   return HISPARSE_OK;
 }
 
@@ -135,7 +175,7 @@ int hisparse_device_bytes(const hisparse_config_t *c, size_t *kv_bytes, size_t *
   if (kv_bytes) *kv_bytes = N * L * (B + 1) * (size_t)c->entry_bytes;
   if (meta_bytes) {
     size_t cap_sum = 0;
-    for (size_t r = 0; r < N; ++r) cap_sum += (size_t)c->capacity[r];
+    for (size_t r = 0; r < N; ++r) cap_sum += (size_t)p2s_stride(c->capacity[r]);
     *meta_bytes = N * G * B * (4 + 4 + 2)          /* slot_pos, last_use, order */
                   + cap_sum * G * 2                 /* page tables */
                   + N * G * k * 4 * 3               /* plan_pos, plan_slot, anchor_out */
@@ -180,7 +220,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   h->init_len.assign(c->init_len, c->init_len + N);
   h->p2s_off.resize(N);
   int64_t off = 0;
-  for (int r = 0; r < N; ++r) { h->p2s_off[r] = off; off += h->cap[r] * G; }
+  for (int r = 0; r < N; ++r) { h->p2s_off[r] = off; off += p2s_stride(h->cap[r]) * G; }
   h->p2s_total = off;
   d.uni_cap = h->cap[0];
   d.uni_init_len = h->init_len[0];
@@ -193,36 +233,43 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) return fail(HISPARSE_ECUDA);
   h->sm_count = sm_count;
   if (cudaFuncSetAttribute(gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
-  // Block size.  One 1024-thread block per SM gives a request the whole SM and all of its shared memory for the
-  // fetch ring.  When the grid takes several waves anyway (more blocks than SMs), two 512-thread blocks per SM hide
-  // each other's dependent trips to memory; each then gets half of the SM's shared memory.
   int want = c->ctas_per_request;
   if (!want) {
     want = 1;
     while (want < 8 && N * want < 32) want <<= 1;
   }
-  d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
-  const int64_t budget_small = smem_per_sm / 2 - 1024 - 256;   // per block: 1 KB reserved by the system, static arrays
-  const bool fits_small = B <= 16 * kThreadsSmall && k <= 4 * kThreadsSmall &&
-                          budget_small - d.meta_smem - kBarBytes >= std::min<int64_t>(d.E, 8192) * 8;
-  if ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) && ((c->flags & HISPARSE_FLAG_WIDE_BLOCKS) || !fits_small)) return fail(HISPARSE_EINVAL);
-  const bool small = fits_small && !(c->flags & HISPARSE_FLAG_WIDE_BLOCKS) &&
-                     ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) || (int64_t)N * want > sm_count);
-  h->T = small ? kThreadsSmall : kThreads;
-  const int64_t budget = small ? budget_small : (int64_t)max_optin - 1024;
-  // shared memory: metadata arrays, one mbarrier per thread, then the staging ring of the fetch pipeline,
-  // which takes whatever is left (pieces of at most 8 KB; at least one piece must fit)
-  const int64_t ring_room = budget - d.meta_smem - kBarBytes;
-  if (ring_room < 16) return fail(HISPARSE_EINVAL);
-  d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
-  const int slots = (int)(ring_room / d.io_chunk);
-  d.io_threads = std::min(slots, h->T);
-  d.io_depth = std::min(slots / d.io_threads, 8);
-  d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
-  d.io_ppr = (int)((d.E + d.io_chunk - 1) / d.io_chunk);
-  h->resolve_smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
+  // Block size and shared memory.  One 1024-thread block per SM gives a request the whole SM: the table of missing
+  // positions has memory of its own (cleared before the dependency wait) and the fetch ring takes all the rest.
+  // When the grid takes several waves anyway (more blocks than SMs), three or two 512-thread blocks share an SM and
+  // hide each other's dependent trips to memory; the table then borrows the ring's memory and the ring is as large
+  // as a third (half) of the SM allows.
+  const bool coop = want > 1;
+  const int64_t piece = std::min<int64_t>(d.E, 8192);
+  auto try_small = [&](int per_sm) {
+    if (!(B <= 16 * kThreadsSmall && k <= 4 * kThreadsSmall)) return false;
+    layout_smem(d, kThreadsSmall, coop, true);
+    const int64_t budget = smem_per_sm / per_sm - 1024 - 256;   // per block: 1 KB reserved by the system, static arrays
+    const int64_t room = budget - d.meta_smem - d.bar_bytes;
+    return room >= piece * 4 && layout_ring(d, kThreadsSmall, room);
+  };
+  const bool want_small = !(c->flags & HISPARSE_FLAG_WIDE_BLOCKS) &&
+                          ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) || (int64_t)N * want > sm_count);
+  if ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) && (c->flags & HISPARSE_FLAG_WIDE_BLOCKS)) return fail(HISPARSE_EINVAL);
+  h->T = kThreads; h->minb = 1;
+  if (want_small) {
+    const char *env = getenv("HISPARSE_BLOCKS_PER_SM");   // tuning knob: 2 or 3 narrow blocks per SM
+    const int first = env && atoi(env) == 2 ? 2 : 3;
+    for (int per_sm = first; per_sm >= 2 && h->T == kThreads; --per_sm)
+      if (try_small(per_sm)) { h->T = kThreadsSmall; h->minb = per_sm; }
+    if (h->T == kThreads && (c->flags & HISPARSE_FLAG_NARROW_BLOCKS)) return fail(HISPARSE_EINVAL);
+  }
+  if (h->T == kThreads) {
+    layout_smem(d, kThreads, coop, false);
+    if (!layout_ring(d, kThreads, (int64_t)max_optin - 1024 - d.meta_smem - d.bar_bytes)) return fail(HISPARSE_EINVAL);
+  }
+  h->resolve_smem = kernel_smem_bytes(d);
   h->replay_smem = h->resolve_smem;   // same offsets, so that both kernels share the pipeline's geometry
-  const void *kern = resolve_kernel_of(h->T);
+  const void *kern = resolve_kernel_of(h->T, h->minb);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
   if (cudaFuncSetAttribute(replay_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - 1024) != cudaSuccess) return fail(HISPARSE_ECUDA);
 
@@ -246,6 +293,15 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
       if (cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg) == cudaSuccess && nclusters >= N) { h->S = s; break; }
       cudaGetLastError();
     }
+  }
+
+  // A grid of several waves of narrow blocks is launched as ONE resident wave whose blocks loop over the requests.
+  h->clusters = N;
+  if (h->S == 1 && h->T == kThreadsSmall) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, h->T, h->resolve_smem) != cudaSuccess) return fail(HISPARSE_ECUDA);
+    const char *env = getenv("HISPARSE_RESIDENT_WAVE");
+    if (per_sm >= 1 && !(env && atoi(env) == 0)) h->clusters = std::min(N, per_sm * sm_count);
   }
 
 #define HS_TRY(expr) do { int rc_ = (expr); if (rc_) return fail(rc_); } while (0)
@@ -518,7 +574,7 @@ int hisparse_dump_state(hisparse_t *h, int req, int layer, int32_t *slot_pos, ui
   }
   if (pos2slot) {
     std::vector<int16_t> tmp((size_t)h->cap[req]);
-    HS_CUDA(cudaMemcpy(tmp.data(), h->d.pos2slot + h->p2s_off[req] + (int64_t)g * h->cap[req], (size_t)h->cap[req] * 2,
+    HS_CUDA(cudaMemcpy(tmp.data(), h->d.pos2slot + h->p2s_off[req] + (int64_t)g * p2s_stride(h->cap[req]), (size_t)h->cap[req] * 2,
                        cudaMemcpyDeviceToHost));
     for (int64_t i = 0; i < h->cap[req]; ++i) pos2slot[i] = tmp[(size_t)i];
   }
@@ -570,7 +626,7 @@ int hisparse_load_state(hisparse_t *h, int req, int layer, const int32_t *slot_p
   HS_CUDA(cudaMemcpy(h->d.slot_pos + rg * B, slot_pos, (size_t)B * 4, cudaMemcpyHostToDevice));
   HS_CUDA(cudaMemcpy(h->d.last_use + rg * B, last_use, (size_t)B * 4, cudaMemcpyHostToDevice));
   HS_CUDA(cudaMemcpy(h->d.order + rg * B, order.data(), (size_t)B * 2, cudaMemcpyHostToDevice));
-  HS_CUDA(cudaMemcpy(h->d.pos2slot + h->p2s_off[req] + (int64_t)g * cap, p2s.data(), (size_t)cap * 2, cudaMemcpyHostToDevice));
+  HS_CUDA(cudaMemcpy(h->d.pos2slot + h->p2s_off[req] + (int64_t)g * p2s_stride(cap), p2s.data(), (size_t)cap * 2, cudaMemcpyHostToDevice));
   HS_CUDA(cudaMemcpy(h->d.t + rg, &resolves, 4, cudaMemcpyHostToDevice));
   if (h->d.order_t) HS_CUDA(cudaMemcpy(h->d.order_t + rg, &resolves, 4, cudaMemcpyHostToDevice));  // the list is current
   const int32_t zero = 0;

@@ -57,7 +57,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
     HS_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
     int optin = 0;
     HS_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    HS_CUDA(cudaFuncSetAttribute(resolve_kernel<kThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 1024));
+    HS_CUDA(cudaFuncSetAttribute(resolve_kernel<kThreads, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - 1024));
     g_noalloc_optin[dev] = optin;
     g_noalloc_ptr[dev] = static_cast<unsigned char *>(p);
   }
@@ -89,16 +89,9 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   d.status = status_dev ? status_dev : reinterpret_cast<uint32_t *>(scratch + 2 * kNoAllocPlanBytes + 3 * kNoAllocCounterBytes);
   d.ticket = nullptr;
   d.phase_ns = nullptr;      // only touched with PHASE_TIMERS, which is off here
-  d.meta_smem = (int)((resolve_smem_bytes(B, k) + 127) & ~(size_t)127);
-  const int64_t ring_room = (int64_t)optin - 1024 - d.meta_smem - kBarBytes;
-  if (ring_room < 16) return HISPARSE_EINVAL;
-  d.io_chunk = (int)std::min<int64_t>(std::min<int64_t>(d.E, 8192), ring_room & ~(int64_t)15);
-  const int slots = (int)(ring_room / d.io_chunk);
-  d.io_threads = std::min(slots, kThreads);
-  d.io_depth = std::min(slots / d.io_threads, 8);
-  d.ring_bytes = d.io_threads * d.io_depth * d.io_chunk;
-  d.io_ppr = (int)((d.E + d.io_chunk - 1) / d.io_chunk);
-  const size_t smem = (size_t)d.meta_smem + kBarBytes + (size_t)d.ring_bytes;
+  layout_smem(d, kThreads, true, false);   // a request's two blocks may share the page-table lookups
+  if (!layout_ring(d, kThreads, (int64_t)optin - 1024 - d.meta_smem - d.bar_bytes)) return HISPARSE_EINVAL;
+  const size_t smem = kernel_smem_bytes(d);
 
   cudaStream_t s = as_stream(stream);
   // the counters other blocks read must not carry the previous call's values into this one
@@ -114,7 +107,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreads>, d, 0, sel_dev, slot_table_dev, hits_dev, misses_dev, S));
+  HS_CUDA(cudaLaunchKernelEx(&cfg, resolve_kernel<kThreads, 1, false>, d, 0, sel_dev, slot_table_dev, hits_dev, misses_dev, S));
   return HISPARSE_OK;
 }
 

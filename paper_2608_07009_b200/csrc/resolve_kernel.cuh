@@ -290,106 +290,201 @@ __device__ __forceinline__ void rebuild_order(const int B, const int W, const ui
   __syncthreads();
 }
 
-// Everything the first block of a cluster does before the fetch can start: Phases 1-2 of Sec. 3.4 and the list of
-// misses.  KPT = row entries per thread (k <= KPT * T).  On return s_plan_pos[i] holds the position of the i-th miss,
-// s_out[j] the slot of every row entry that hit (or -1, a duplicate marker, or the rank of its miss), s_hitbits the
-// hit marks and s_order the staged recency list; `fast` = nothing missed (and the list may be left behind).
-template <int T, int IPT, int KPT>
-__device__ __forceinline__ void resolve_metadata(const DevState &d, const int r, const int64_t rg, const int32_t *row,
-                                                 int32_t *s_sel, int32_t *s_out, int32_t *s_plan_pos,
-                                                 int32_t *s_plan_slot, unsigned long long *s_tab, uint32_t *s_hitbits,
-                                                 uint32_t *s_vicbits, uint16_t *s_order, int *s_warp, int *s_misc,
-                                                 const int64_t cap_r, const int64_t init_len_r,
-                                                 const int64_t p2s_off_r, unsigned long long *stamps,
-                                                 unsigned char *s_ring, unsigned long long *s_bars,
-                                                 const uint32_t t_now, int *s_warp_pre, int16_t *s_got, const int S,
-                                                 int &m, uint32_t &my_status, bool &fast) {
-  const int tid = threadIdx.x;
-  const int k = d.k, B = d.B, H = d.H;
-  const uint32_t mask = (uint32_t)(H - 1);
-  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
-  bool timed_out = false;
+// What a block needs from shared memory, carved out of the dynamic allocation by the offsets fixed at create.
+struct SmemView {
+  int32_t *sel;                  // the selected row; once consumed, its space holds the recency list (`order`)
+  uint16_t *order;
+  int32_t *plan_pos, *plan_slot;
+  uint16_t *missj;
+  uint8_t *marks;                // one byte per slot: == the request's tag when a selection hit the slot
+  uint32_t *hitbits, *vicbits;   // hit marks as a bitset (built from `marks` once something missed), victim marks
+  int32_t *hitpre, *vicpre;
+  int *hist;
+  int16_t *got;
+  unsigned long long *tab;
+  unsigned long long *bars;
+  unsigned char *ring;
+  int *warp;                     // 32 ints of scratch for block scans
+  int *misc;                     // two sets used by alternate requests: [0] a missing position was selected twice
+                                 // [1] selections that hit  [2] the newest position was selected  [3] distinct slots hit
+};
 
-  // Phase 1: stage the row and the recency order (one round trip to HBM).  The request's slice of the page
-  // table is streamed into the (still idle) fetch ring with bulk copies when it fits, so that Phase 2's k random
-  // lookups hit shared memory instead of queueing as 32-byte sector reads on one SM.
-  const int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)(rg - (int64_t)r * d.G) * cap_r;
-  const uintptr_t p2s_aligned = (uintptr_t)p2s & ~(uintptr_t)15;
-  const int lead = (int)(((uintptr_t)p2s - p2s_aligned) >> 1);
-  const int64_t stage_bytes = ((int64_t)lead * 2 + cap_r * 2) & ~(int64_t)15;  // whole 16-byte units only
-  const bool staged = stage_bytes + 16 <= (int64_t)d.ring_bytes;
-  const bool coop = !staged && S > 1;  // same decision in every block of the cluster (depends on the request only)
-  if (coop) cluster_arrive_relaxed();  // phase A, see cluster_lookups
-  const uint32_t stage_bar = smem_u32(s_bars + kThreads);
-  const uint16_t *order_g = d.order + rg * B;
-  // 16-byte aligned arrays are fetched by ONE thread with bulk copies (a handful of instructions for the whole
-  // block); anything else falls back to per-thread cp.async
+// `it` = how many requests this block has resolved before the current one (picks the set of flags).
+__device__ __forceinline__ SmemView smem_view(const DevState &d, unsigned char *raw, const int it) {
+  SmemView v;
+  v.sel = reinterpret_cast<int32_t *>(raw);
+  v.order = reinterpret_cast<uint16_t *>(raw);
+  v.plan_pos = reinterpret_cast<int32_t *>(raw + d.sm_plan_pos);
+  v.plan_slot = reinterpret_cast<int32_t *>(raw + d.sm_plan_slot);
+  v.missj = reinterpret_cast<uint16_t *>(raw + d.sm_missj);
+  const int wpad = (d.W + 3) & ~3;
+  v.marks = raw + d.sm_marks;
+  v.hitbits = reinterpret_cast<uint32_t *>(raw + d.sm_bits);
+  v.vicbits = v.hitbits + wpad;
+  v.hitpre = reinterpret_cast<int32_t *>(v.vicbits + wpad);
+  v.vicpre = v.hitpre + wpad;
+  v.hist = reinterpret_cast<int *>(raw + d.sm_hist);
+  v.got = reinterpret_cast<int16_t *>(raw + d.sm_got);
+  v.bars = reinterpret_cast<unsigned long long *>(raw + d.meta_smem);
+  v.ring = raw + d.meta_smem + d.bar_bytes;
+  v.tab = reinterpret_cast<unsigned long long *>(d.sm_tab >= 0 ? raw + d.sm_tab : v.ring);
+  v.warp = reinterpret_cast<int *>(raw + d.sm_misc);
+  v.misc = v.warp + 32 + (it & 1) * 8;
+  return v;
+}
+
+// Where a request's slice of the page table is and whether it can be staged in the (still idle) fetch ring.
+struct SliceGeom {
+  const int16_t *p2s;        // the request's slice (one entry per position)
+  uintptr_t aligned;         // its address rounded down to 16 bytes
+  int lead;                  // entries between `aligned` and p2s
+  int64_t stage_bytes;       // whole 16-byte units that cover the slice
+  bool staged;
+};
+
+__device__ __forceinline__ SliceGeom slice_geom(const DevState &d, const int g, const int64_t cap_r, const int64_t p2s_off_r) {
+  SliceGeom q;
+  q.p2s = d.pos2slot + p2s_off_r + (int64_t)g * p2s_stride(cap_r);
+  q.aligned = (uintptr_t)q.p2s & ~(uintptr_t)15;
+  q.lead = (int)(((uintptr_t)q.p2s - q.aligned) >> 1);
+  q.stage_bytes = ((int64_t)q.lead * 2 + cap_r * 2) & ~(int64_t)15;
+  q.staged = q.stage_bytes + 16 <= (int64_t)d.ring_bytes;
+  return q;
+}
+
+// One request's resolve as a block sees it (block-uniform).
+struct ReqCtx {
+  int r, it, S, layer, g;
+  int64_t rg, cap_r, init_len_r, p2s_off_r;
+  const int32_t *row;
+  int32_t *trow, *arow;
+  int32_t *hits_out, *misses_out;
+  bool has_next;             // the block takes another request after this one
+  int tag;                   // 1..255: what a hit writes into `marks` for this request (so that they need no clearing)
+};
+
+__device__ __forceinline__ void request_geom(const DevState &d, const int r, int64_t &cap_r, int64_t &init_len_r,
+                                             int64_t &p2s_off_r) {
+  const bool uni = d.uni_cap >= 0;  // fixed at create
+  cap_r = uni ? d.uni_cap : d.cap[r];
+  init_len_r = uni ? d.uni_init_len : d.init_len[r];
+  p2s_off_r = uni ? (int64_t)r * d.G * p2s_stride(d.uni_cap) : d.p2s_off[r];
+}
+
+// Phase 1: the row and, when it fits the idle fetch ring, the request's slice of the page table start their way to
+// shared memory as bulk copies issued by the lanes of the first warp, all completing on one mbarrier (`stage_bar`).
+// Staging the slice turns Phase 2's k random lookups into shared-memory reads instead of 32-byte sector reads
+// queueing on one SM.  Called by every thread of the block; shapes that bulk copies cannot take (unaligned row, the
+// last partial 16-byte unit of the slice) are copied by plain loads, which the consumer orders with a block barrier.
+constexpr uint32_t kStagePiece = 16384;  // bytes per bulk copy when a row and a page-table slice are staged (measured:
+                                         // 1 KB pieces make the staging slower, not faster)
+
+template <int T>
+__device__ __forceinline__ void stage_issue(const DevState &d, const SmemView &v, const SliceGeom &q, const int32_t *row,
+                                            const int64_t cap_r, const uint32_t stage_bar) {
+  const int tid = threadIdx.x;
+  const int k = d.k;
   const bool sel_bulk = (((uintptr_t)row | (uintptr_t)(k * 4)) & 15) == 0;
-  const bool ord_bulk = (((uintptr_t)order_g | (uintptr_t)(B * 2)) & 15) == 0;
-  // one expect_tx for everything; each copy is issued by the first lane of a different warp, so that the copies
-  // enter the bulk-copy engine side by side (a copy that lands before the expect_tx only makes the count dip)
-  if (tid == 0) {
-    const uint32_t tx = (sel_bulk ? (uint32_t)k * 4u : 0u) + (ord_bulk ? (uint32_t)B * 2u : 0u) +
-                        (staged ? (uint32_t)stage_bytes : 0u);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(stage_bar), "r"(tx) : "memory");
-    if (sel_bulk)
+  if (tid < 32) {
+    // pieces of kStagePiece bytes, issued side by side by the lanes of the warp
+    const uint32_t row_bytes = sel_bulk ? (uint32_t)k * 4u : 0u, slice_bytes = q.staged ? (uint32_t)q.stage_bytes : 0u;
+    if (tid == 0)  // (a copy that lands before this arrival only makes the byte count dip: the phase cannot complete before it)
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(stage_bar), "r"(row_bytes + slice_bytes) : "memory");
+    const uint32_t row_pieces = (row_bytes + kStagePiece - 1) / kStagePiece, slice_pieces = (slice_bytes + kStagePiece - 1) / kStagePiece;
+    for (uint32_t p = (uint32_t)tid; p < row_pieces + slice_pieces; p += 32u) {
+      const bool in_row = p < row_pieces;
+      const uint32_t o = (in_row ? p : p - row_pieces) * kStagePiece, total = in_row ? row_bytes : slice_bytes;
+      const uint32_t n = total - o < kStagePiece ? total - o : kStagePiece;
+      const uint32_t dst = (in_row ? smem_u32(v.sel) : smem_u32(v.ring)) + o;
+      const char *src = (in_row ? reinterpret_cast<const char *>(row) : reinterpret_cast<const char *>(q.aligned)) + o;
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(s_sel)), "l"(row), "r"((uint32_t)k * 4u), "r"(stage_bar) : "memory");
-  }
-  if (tid == 32 && ord_bulk)
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(s_order)), "l"(order_g), "r"((uint32_t)B * 2u), "r"(stage_bar) : "memory");
-  if (staged && tid >= 64 && (tid & 31) == 0) {
-    constexpr int kPiece = 16384;
-    for (int64_t o = (int64_t)((tid >> 5) - 2) * kPiece; o < stage_bytes; o += (int64_t)(T / 32 - 2) * kPiece) {
-      const uint32_t n = (uint32_t)(stage_bytes - o < kPiece ? stage_bytes - o : kPiece);
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(s_ring) + (uint32_t)o), "l"((const char *)p2s_aligned + o), "r"(n), "r"(stage_bar) : "memory");
+                   ::"r"(dst), "l"(src), "r"(n), "r"(stage_bar) : "memory");
     }
   }
-  if (!sel_bulk) stage_async(s_sel, row, k * 4);
-  if (!ord_bulk) stage_async(s_order, order_g, B * 2);
-  if (staged && tid >= 32 && tid < 40) {  // the last, partial 16-byte unit of the slice: plain copies
-    const int64_t e = stage_bytes / 2 + (tid - 32);
-    if (e < lead + cap_r) reinterpret_cast<int16_t *>(s_ring)[e] = reinterpret_cast<const int16_t *>(p2s_aligned)[e];
+  if (!sel_bulk) stage_async(v.sel, row, k * 4);
+  if (q.staged && tid >= 32 && tid < 40) {  // the last, partial 16-byte unit of the slice: plain copies
+    const int64_t e = q.stage_bytes / 2 + (tid - 32);
+    if (e < q.lead + cap_r) reinterpret_cast<int16_t *>(v.ring)[e] = reinterpret_cast<const int16_t *>(q.aligned)[e];
   }
+}
+
+// Phase 2 of Sec. 3.4 as the first block of a cluster runs it, up to the block-wide vote "did anything miss?".
+// Thread t owns the KPT consecutive row entries [t*KPT, t*KPT + KPT): it reads them with one vector load, looks them
+// up in the page table, marks the slots that hit, and writes its part of the slot table at once (a hit's slot is final;
+// an entry that missed gets its slot later, a placeholder for now).  On return pos[] / cls[] hold the thread's
+// positions and their classification (slot, B for the newest record, kMiss, or -1), `any_miss` the vote.
+// `stage_parity` = phase of the staging barrier that stage_issue's copies for this request complete.
+template <int T, int KPT>
+__device__ __forceinline__ void lookup_phase(const DevState &d, const SmemView &v, const SliceGeom &q, const ReqCtx &c,
+                                             const uint32_t stage_parity, unsigned long long *stamps,
+                                             int32_t (&pos)[KPT], int32_t (&cls)[KPT], uint32_t &my_status, bool &any_miss,
+                                             uint32_t &t_now, uint32_t &order_t) {
+  const int tid = threadIdx.x;
+  const int k = d.k, B = d.B;
+  const int r = c.r, S = c.S;
+  const int64_t rg = c.rg, cap_r = c.cap_r, init_len_r = c.init_len_r;
+  const int32_t *row = c.row;
+  int32_t *trow = c.trow, *arow = c.arow;
+  int *s_misc = v.misc;
+  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+  const bool coop = !q.staged && S > 1;  // same decision in every block of the cluster (depends on the request only)
+  if (coop) cluster_arrive_relaxed();    // phase A, see cluster_lookups
+  const uint32_t stage_bar = smem_u32(v.bars + T);
+  const bool sel_bulk = (((uintptr_t)row | (uintptr_t)(k * 4)) & 15) == 0;
+  // the scalars of this resolve, loaded while the copies fly
   const int64_t na = *(volatile int32_t *)d.n_appends;
+  t_now = d.t[rg] + 1u;
+  order_t = d.order_t ? d.order_t[rg] : t_now - 1u;  // resolve count the recency list is current for
   const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
   const int64_t newest = (na > 0 && init_len_r + na <= cap_r) ? init_len_r + na - 1 : -1;
   if (timers && tid == 0) stamps[8] = clock64();
-  if (!sel_bulk || !ord_bulk) asm volatile("cp.async.wait_all;" ::: "memory");
-  bool use_staged = staged;
-  if (!mbar_wait_bounded(stage_bar, 0u)) {
-    // bounded wait expired: the row cannot be trusted either, so this request resolves nothing in this launch
-    use_staged = false;
-    my_status |= HISPARSE_STATUS_TIMEOUT;
-    timed_out = true;
+  if (!sel_bulk) asm volatile("cp.async.wait_all;" ::: "memory");
+  // One warp waits for the copies; the others wait for that warp at a block barrier, which costs no issue slots (a
+  // block-wide spin on the mbarrier was measured to take most of the instructions of a resolve in which nothing
+  // misses, at the expense of the other blocks on the SM).  The barrier also orders the plain copies above.
+  bool landed = true;
+  if (tid < 32 && !mbar_wait_bounded(stage_bar, stage_parity)) {
+    // bounded wait expired: the row cannot be trusted either, so this request resolves nothing in this launch.  The
+    // copies get one more bounded chance to land before anything else uses (or the block gives up) their memory.
+    mbar_wait_bounded(stage_bar, stage_parity);
+    landed = false;
   }
-  __syncthreads();
+  const bool timed_out = __syncthreads_or(!landed) != 0;
+  const bool use_staged = q.staged && !timed_out;
+  if (timed_out) my_status |= HISPARSE_STATUS_TIMEOUT;
   if (timers && tid == 0) stamps[9] = clock64();
-  const int16_t *s_p2s = reinterpret_cast<const int16_t *>(s_ring) + lead;
-  if (coop) cluster_lookups<T>(row, p2s, k, len, 0, S, s_got);
+  const int16_t *s_p2s = reinterpret_cast<const int16_t *>(v.ring) + q.lead;
+  if (coop) cluster_lookups<T>(row, q.p2s, k, len, 0, S, v.got);
 
-  // Phase 2: hit detection through the page table (position -> slot): all of a thread's lookups are issued
-  // before the first is used.  Hits keep their slot and are stamped first; the selections that are not
-  // resident go into the hash table (position -> row index), whose only job is to catch a position that is
-  // selected twice, so that it claims one victim, not two.
-  int32_t pos[KPT], got[KPT];
+  // Phase 2: hit detection through the page table (position -> slot); all of a thread's lookups are issued
+  // before the first is used.
+  const int j0 = tid * KPT;
+#pragma unroll
+  for (int i = 0; i < KPT; ++i) pos[i] = -1;
+  if (j0 < k && !timed_out) {
+    if constexpr (KPT == 4) {
+      const int4 x = *reinterpret_cast<const int4 *>(v.sel + j0);
+      pos[0] = x.x; pos[1] = x.y; pos[2] = x.z; pos[3] = x.w;
+    } else {
+      const int2 x = *reinterpret_cast<const int2 *>(v.sel + j0);
+      pos[0] = x.x; pos[1] = x.y;
+    }
+  }
+  int32_t got[KPT];
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
-    const int j = tid + i * T;
-    pos[i] = (j < k && !timed_out) ? s_sel[j] : -1;
+    if (j0 + i >= k) pos[i] = -1;
     const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
     if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
     if (!ok) pos[i] = -1;
-    got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : coop ? s_got[j] : __ldg(p2s + pos[i]));
+    got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : coop ? v.got[j0 + i] : __ldg(q.p2s + pos[i]));
   }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring goes back to the bulk-copy engine later
-  int any_miss = 0;
+  int miss = 0, nhit = 0;
+  int32_t val[KPT];
+  const int32_t base = r * (B + 1);
+  const uint8_t tag = (uint8_t)c.tag;
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
-    const int j = tid + i * T;
-    if (j >= k) break;
     const int32_t p = pos[i];
     int32_t o = -1;
     if (p >= 0) {
@@ -397,92 +492,144 @@ __device__ __forceinline__ void resolve_metadata(const DevState &d, const int r,
         o = B;
         if (atomicExch(&s_misc[2], 1) != 0) my_status |= HISPARSE_STATUS_DUPLICATE;
       } else if (got[i] >= 0) {
-        const int s = got[i];
-        o = s;
-        const uint32_t bit = 1u << (s & 31);
-        // a bit that is already set = the same resident position selected again: same slot, counted once.
-        // The hit's stamp is written later, in slot order (coalesced), from the hit bits.
-        if (atomicOr(&s_hitbits[s >> 5], bit) & bit) my_status |= HISPARSE_STATUS_DUPLICATE;
+        // A plain byte store marks the slot (shared-memory atomics on a bitset were measured to take about half of
+        // a resolve in which nothing misses).  The hit's stamp is written later, in slot order (coalesced), from
+        // the marks; a resident position selected twice marks one slot twice, which the counts reveal.
+        o = got[i];
+        v.marks[o] = tag;
+        ++nhit;
       } else {
         o = kMiss;
-        any_miss = 1;
-        const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)j;
-        uint32_t h = hash_pos(p, d.hshift);
-        for (uint32_t it = 0; it <= mask; ++it) {
-          const unsigned long long old = atomicCAS(&s_tab[h], kEmptyEntry, entry);
-          if (old == kEmptyEntry) break;
-          if ((int32_t)(old >> 32) == p) {  // selected twice: the lowest row index owns the entry
-            atomicMin(&s_tab[h], entry);
-            s_misc[0] = 1;
-            break;
-          }
-          h = (h + 1u) & mask;
-        }
+        miss = 1;
       }
     }
-    s_out[j] = o;
+    cls[i] = o;
+    val[i] = o < 0 ? -1 : base + o;
   }
-  any_miss = __syncthreads_or(any_miss);
-  if (!any_miss && d.order_t != nullptr) {
-    // Nothing to fetch, no victim to choose: the caller writes the table and stamps the hits, and the recency list
-    // is left as it is (rebuild_order brings it up to date in the next resolve that needs victims).
-    fast = true;
-    m = 0;
-    return;
+  // Phase 5, first part: the thread's entries of the slot table (and of the group's shared table), one vector store
+  const bool vec = (((uintptr_t)trow | (uintptr_t)arow) & (KPT * 4 - 1)) == 0 && j0 + KPT <= k;
+  if (vec) {
+    if constexpr (KPT == 4) {
+      *reinterpret_cast<int4 *>(trow + j0) = make_int4(val[0], val[1], val[2], val[3]);
+      if (arow) *reinterpret_cast<int4 *>(arow + j0) = make_int4(cls[0] < 0 ? -1 : cls[0], cls[1] < 0 ? -1 : cls[1],
+                                                                 cls[2] < 0 ? -1 : cls[2], cls[3] < 0 ? -1 : cls[3]);
+    } else {
+      *reinterpret_cast<int2 *>(trow + j0) = make_int2(val[0], val[1]);
+      if (arow) *reinterpret_cast<int2 *>(arow + j0) = make_int2(cls[0] < 0 ? -1 : cls[0], cls[1] < 0 ? -1 : cls[1]);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < KPT; ++i)
+      if (j0 + i < k) {
+        trow[j0 + i] = val[i];
+        if (arow) arow[j0 + i] = cls[i] < 0 ? -1 : cls[i];
+      }
   }
+  nhit = __reduce_add_sync(0xffffffffu, nhit);
+  if ((tid & 31) == 0 && nhit) atomicAdd(&s_misc[1], nhit);
+  any_miss = __syncthreads_or(miss) != 0;
   if (timers && tid == 0) stamps[10] = clock64();
+}
+
+// The rest of what precedes the fetch when something missed: the missing positions go through a table (position ->
+// row index) whose only job is to catch a position that was selected twice, so that it claims one victim, not two;
+// then ONE block scan puts the misses in selection order.  On return plan_pos[i] / missj[i] hold the position and
+// the row index of the i-th miss and m their number.
+template <int T, int KPT>
+__device__ __forceinline__ void list_misses(const DevState &d, const SmemView &v, int32_t *trow, int32_t *arow,
+                                            unsigned long long *stamps, int *s_misc,
+                                            const int32_t (&pos)[KPT], int32_t (&cls)[KPT], uint32_t &my_status, int &m) {
+  const int tid = threadIdx.x;
+  const int H = d.H;
+  const uint32_t mask = (uint32_t)(H - 1);
+  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+  const int j0 = tid * KPT;
+  if (d.sm_tab < 0) {  // the table shares the ring's memory and is cleared only now that it is needed
+    for (int i = tid; i < H; i += T) v.tab[i] = kEmptyEntry;
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < KPT; ++i)
+    if (cls[i] == kMiss) {
+      const int32_t p = pos[i];
+      const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)(j0 + i);
+      uint32_t h = hash_pos(p, d.hshift);
+      for (uint32_t it = 0; it <= mask; ++it) {
+        const unsigned long long old = atomicCAS(&v.tab[h], kEmptyEntry, entry);
+        if (old == kEmptyEntry) break;
+        if ((int32_t)(old >> 32) == p) {  // selected twice: the lowest row index owns the entry
+          atomicMin(&v.tab[h], entry);
+          s_misc[0] = 1;
+          break;
+        }
+        h = (h + 1u) & mask;
+      }
+    }
+  __syncthreads();
+  if (timers && tid == 0) stamps[11] = clock64();
   if (s_misc[0]) {  // rare: every later occurrence of a repeated missing position follows the first one
-    for (int j = tid; j < k; j += T) {
-      if (s_out[j] == kMiss) {
-        const int32_t key[1] = {s_sel[j]};
+#pragma unroll
+    for (int i = 0; i < KPT; ++i)
+      if (cls[i] == kMiss) {
+        const int32_t key[1] = {pos[i]};
         int32_t owner[1];
-        table_lookup<1>(s_tab, mask, d.hshift, key, owner);
-        if (owner[0] != j) {
-          s_out[j] = kDupBase - owner[0];
+        table_lookup<1>(v.tab, mask, d.hshift, key, owner);
+        if (owner[0] != j0 + i) {
+          cls[i] = -1;  // not a miss of its own; its table entry is copied from the owner's at the end
+          trow[j0 + i] = kDupBase - owner[0];
+          if (arow) arow[j0 + i] = kDupBase - owner[0];
           my_status |= HISPARSE_STATUS_DUPLICATE;
         }
       }
-    }
-    __syncthreads();
   }
-  if (timers && tid == 0) stamps[11] = clock64();
-
-  // Phase 3, first half: the misses in selection order (one block scan; thread t owns KPT consecutive row entries).
-  // Their positions are all the fetch needs to start loading; the victims are only needed when a record is stored.
-  {
-    uint32_t miss_mask = 0;
+  // Phase 3, first half: the misses in selection order.  Their positions are all the fetch needs to start loading;
+  // the victims are only needed when a record is stored.
+  uint32_t miss_mask = 0;
 #pragma unroll
-    for (int i = 0; i < KPT; ++i) {
-      const int j = tid * KPT + i;
-      if (j < k && s_out[j] == kMiss) miss_mask |= 1u << i;
+  for (int i = 0; i < KPT; ++i)
+    if (cls[i] == kMiss) miss_mask |= 1u << i;
+  int mrank = block_scan_excl(__popc(miss_mask), v.warp, m);
+#pragma unroll
+  for (int i = 0; i < KPT; ++i)
+    if ((miss_mask >> i) & 1u) {
+      v.plan_pos[mrank] = pos[i];
+      v.missj[mrank] = (uint16_t)(j0 + i);
+      ++mrank;
     }
-    int mrank = block_scan_excl(__popc(miss_mask), s_warp, m);
-#pragma unroll
-    for (int i = 0; i < KPT; ++i)
-      if ((miss_mask >> i) & 1u) {
-        const int j = tid * KPT + i;
-        s_plan_pos[mrank] = s_sel[j];      // position of the mrank-th miss
-        s_out[j] = kRankBase - mrank;      // its slot is the mrank-th victim, looked up when the table is written
-        ++mrank;
-      }
-  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the table's memory may be the ring
   if (timers && tid == 0) stamps[12] = clock64();
   __syncthreads();
 }
 
-// Phase 3, second half (runs while the first loads are in flight): brings the recency list up to date if it lags,
-// then ONE block scan over the non-hit slots in recency order.  Thread t owns IPT consecutive entries of the list.
-// On return s_plan_slot[i] holds the victim of the i-th miss, s_vicbits the victims' marks, s_order the untouched
-// slots compacted at its front and n_nonhit the number of slots without a hit.
+// Phase 3, second half (runs while the first loads are in flight): waits for the recency list (its load was issued
+// right after the vote, into the memory the row had used), brings it up to date if it lags, then ONE block scan over
+// the non-hit slots in recency order.  Thread t owns IPT consecutive entries of the list.  On return plan_slot[i] holds
+// the victim of the i-th miss, vicbits the victims' marks, order the untouched slots compacted at its front and
+// n_nonhit the number of slots without a hit.
 template <int T, int IPT>
-__device__ __forceinline__ void choose_victims(const DevState &d, const int r, const int64_t rg, const int m,
-                                               int32_t *s_plan_slot, unsigned long long *s_tab, const uint32_t *s_hitbits,
-                                               uint32_t *s_vicbits, uint16_t *s_order, int *s_warp, int *s_warp_pre,
-                                               unsigned long long *stamps, const uint32_t t_now, const uint32_t order_t,
-                                               int &n_nonhit) {
+__device__ __forceinline__ void choose_victims(const DevState &d, const SmemView &v, const int r, const int64_t rg,
+                                               const int m, unsigned long long *stamps, const uint32_t t_now,
+                                               const uint32_t order_t, const bool order_bulk, const uint32_t order_parity,
+                                               uint32_t &my_status, int &n_nonhit) {
   const int tid = threadIdx.x;
   const int B = d.B;
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+  int32_t *s_plan_slot = v.plan_slot;
+  uint32_t *s_hitbits = v.hitbits, *s_vicbits = v.vicbits;
+  uint16_t *s_order = v.order;
+  int *s_warp_pre = v.vicpre;
+  int *s_warp = v.warp;
+  if (order_bulk) {  // one warp waits for the copy, the others for that warp (see lookup_phase)
+    bool landed = true;
+    if (tid < 32 && !mbar_wait_bounded(smem_u32(v.bars + T + 1), order_parity)) {
+      mbar_wait_bounded(smem_u32(v.bars + T + 1), order_parity);
+      landed = false;
+    }
+    if (__syncthreads_or(!landed)) my_status |= HISPARSE_STATUS_TIMEOUT;
+  } else {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncthreads();
+  }
   if (order_t != t_now - 1u) {
     const uint32_t *last_use = d.last_use + rg * B;
     rebuild_order<T, IPT>(B, d.W, last_use, 2u * order_t + 2u, t_now - 1u - order_t, s_order, s_vicbits, s_warp_pre, s_warp);
@@ -534,7 +681,7 @@ __device__ __forceinline__ void choose_victims(const DevState &d, const int r, c
       // RANDOM: victims by hashed key, paired with the misses in ascending slot order; the list is kept as for LRU
       __syncthreads();
       const unsigned long long base = mix64(d.policy_seed ^ (((unsigned long long)(uint32_t)r << 32) | (uint32_t)(rg - (int64_t)r * d.G)));
-      select_random_victims<IPT>(B, m, base, t_now, s_hitbits, s_vicbits, reinterpret_cast<int *>(s_tab), s_warp);
+      select_random_victims<IPT>(B, m, base, t_now, s_hitbits, s_vicbits, v.hist, s_warp);
       uint32_t keep = 0;
 #pragma unroll
       for (int i = 0; i < IPT; ++i)
@@ -573,191 +720,101 @@ __device__ __forceinline__ void choose_victims(const DevState &d, const int r, c
   if (timers && tid == 0) stamps[14] = clock64();
 }
 
-template <int T>
-__global__ void __launch_bounds__(T, kThreads / T)
-resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ sel, int32_t *__restrict__ table,
-               int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out, const int S) {
+// Everything the first block of a cluster does for a request in which something missed (or whose recency list is kept
+// current by every resolve): list the misses, start the fetch, choose the victims while the first loads fly, write the
+// metadata back, rewrite the recency list, then drain the fetch.  pos / cls come from lookup_phase.
+template <int T, int KPT>
+__device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, const int32_t (&pos)[KPT],
+                                          int32_t (&cls)[KPT], const uint32_t t, const uint32_t order_t,
+                                          uint32_t my_status, uint32_t &fetch_parity, uint32_t &order_parity,
+                                          bool &gave_up) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ int s_warp[32];
-  __shared__ int s_misc[4];  // [0] a missing position was selected twice  [2] the newest position was selected
+  const SmemView v = smem_view(d, smem_raw, c.it);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int r = blockIdx.x / S, part = blockIdx.x - r * S;
-  const int g = layer / d.lpg;
-  const int k = d.k, B = d.B, H = d.H, W = d.W;
-  const int64_t rg = (int64_t)r * d.G + g;
+  const int k = d.k, B = d.B, W = d.W, S = c.S, r = c.r;
+  const int64_t rg = c.rg;
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
   unsigned long long *stamps = d.phase_ns + (int64_t)r * 16;
-
-  unsigned long long *s_tab = reinterpret_cast<unsigned long long *>(smem_raw);
-  int32_t *s_sel = reinterpret_cast<int32_t *>(s_tab + H);
-  int32_t *s_out = s_sel + k;
-  int32_t *s_plan_pos = s_out + k;        // first the row indices of the misses, then their positions
-  int32_t *s_plan_slot = s_plan_pos + k;  // victims, in order
-  uint32_t *s_hitbits = reinterpret_cast<uint32_t *>(s_plan_slot + k);
-  uint32_t *s_vicbits = s_hitbits + W;
-  int32_t *s_hitpre = reinterpret_cast<int32_t *>(s_vicbits + W);
-  int32_t *s_vicpre = s_hitpre + W;
-  uint16_t *s_order = reinterpret_cast<uint16_t *>(s_vicpre + W);
-  int16_t *s_got = reinterpret_cast<int16_t *>(s_order + ((B + 7) & ~7));  // page-table answers from the whole cluster
-  unsigned long long *s_bars = reinterpret_cast<unsigned long long *>(smem_raw + d.meta_smem);
-  unsigned char *s_ring = smem_raw + d.meta_smem + kBarBytes;
-
-  // Prologue that depends on nothing an earlier kernel wrote: barriers, cleared marks and table.  With
-  // programmatic dependent launch it overlaps the tail of whatever runs before this kernel in the stream.
-  fetch_barriers_init(s_bars, d.io_threads);
-  if (part == 0) {
-    for (int i = tid; i < H; i += T) s_tab[i] = kEmptyEntry;
-    for (int i = tid; i < W; i += T) { s_hitbits[i] = 0u; s_vicbits[i] = 0u; }
-    if (tid < 4) s_misc[tid] = 0;
-  }
-  const bool uni = d.uni_cap >= 0;  // fixed at create
-  const int64_t cap_r = uni ? d.uni_cap : d.cap[r], init_len_r = uni ? d.uni_init_len : d.init_len[r],
-                p2s_off_r = uni ? (int64_t)r * d.G * d.uni_cap : d.p2s_off[r];
-  if (part == 0 && tid < 3) {
-    // Warm L2 with what Phase 1 will stage (row, recency order, page-table slice).  A prefetch consumes nothing, and
-    // L2 is where earlier kernels' writes land, so this is safe before the dependency wait; when the previous kernel
-    // lets its dependents start early, the staging after the wait then reads L2 instead of HBM.
-    const char *p = tid == 0 ? reinterpret_cast<const char *>(sel + (int64_t)r * k)
-                  : tid == 1 ? reinterpret_cast<const char *>(d.order + rg * B)
-                             : reinterpret_cast<const char *>(d.pos2slot + p2s_off_r + (int64_t)g * cap_r);
-    int64_t n = tid == 0 ? (int64_t)k * 4 : tid == 1 ? (int64_t)B * 2 : cap_r * 2;
-    const uintptr_t a = ((uintptr_t)p + 15) & ~(uintptr_t)15;   // whole 16-byte units inside the array only
-    n = (n - (int64_t)(a - (uintptr_t)p)) & ~(int64_t)15;
-    if (n > (1 << 20)) n = 1 << 20;                             // no point warming more than the ring could stage
-    if (n > 0)
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a), "r"((uint32_t)n) : "memory");
-  }
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (part != 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  TmaFetch fetch;
-  fetch.active = false;
+  int *s_misc = v.misc;
   int m = 0, n_nonhit = 0;
-  uint32_t t = 0;
-  bool fast = false;  // first block only: no selection missed, the short path below was taken
-  if (part != 0) {
-    // same test as in resolve_metadata: is this request's page-table slice too large to be staged?
-    const int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
-    const int lead = (int)((((uintptr_t)p2s) & 15) >> 1);
-    const int64_t stage_bytes = ((int64_t)lead * 2 + cap_r * 2) & ~(int64_t)15;
-    if (!(stage_bytes + 16 <= (int64_t)d.ring_bytes)) {
-      const int64_t na = *(volatile int32_t *)d.n_appends;
-      const int64_t len = init_len_r + na < cap_r ? init_len_r + na : cap_r;
-      cluster_arrive_relaxed();  // phase A
-      cluster_lookups<T>(sel + (int64_t)r * k, p2s, k, len, part, S, s_got);
-    }
+  for (int i = tid; i < W; i += T) v.vicbits[i] = 0u;  // ordered before their first use by list_misses' barriers
+  // the hit marks as a bitset, which the victim choice and the list rewrite work on (every mark was written before
+  // the vote; the loop bound is uniform, so every lane takes part in the ballot)
+  for (int sb = 0; sb < B; sb += T) {
+    const int s = sb + tid;
+    const uint32_t word = __ballot_sync(0xffffffffu, s < B && v.marks[s] == (uint8_t)c.tag);
+    if (lane == 0 && (s >> 5) < W) v.hitbits[s >> 5] = word;
   }
-  if (part == 0) {
-    if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
-    t = d.t[rg] + 1u;
-    const uint32_t order_t = d.order_t ? d.order_t[rg] : t - 1u;  // resolve count the recency list is current for
-    const uint32_t miss_stamp = 2u * t;
-    uint32_t my_status = 0;
-    const int32_t *row = sel + (int64_t)r * k;
-#define HS_META(IPT, KPT)                                                                                         \
-  resolve_metadata<T, IPT, KPT>(d, r, rg, row, s_sel, s_out, s_plan_pos, s_plan_slot, s_tab, s_hitbits, s_vicbits,     \
-                             s_order, s_warp, s_misc, cap_r, init_len_r, p2s_off_r, stamps, s_ring, s_bars, t,      \
-                             s_vicpre, s_got, S, m, my_status, fast)
-    if constexpr (T == kThreads) {
-      if (k <= 2 * T) {
-        if (B <= 4 * T) HS_META(4, 2);
-        else if (B <= 8 * T) HS_META(8, 2);
-        else HS_META(16, 2);
-      } else {
-        if (B <= 4 * T) HS_META(4, kSelPerThread);
-        else if (B <= 8 * T) HS_META(8, kSelPerThread);
-        else HS_META(16, kSelPerThread);
-      }
-    } else {  // the small block is only chosen for B <= 16 T and k <= 4 T
-      if (B <= 8 * T) HS_META(8, 4);
-      else HS_META(16, 4);
+  // The recency list starts its way into the memory the row occupied (every thread consumed its row entries before
+  // the vote); it is needed only once the first loads are in flight.
+  const uint16_t *order_g = d.order + rg * B;
+  const bool order_bulk = (((uintptr_t)order_g | (uintptr_t)(B * 2)) & 15) == 0;
+  if (order_bulk) {
+    if (tid == 0) {
+      const uint32_t bar = smem_u32(v.bars + T + 1);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)B * 2u) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(v.order)), "l"(order_g), "r"((uint32_t)B * 2u), "r"(bar) : "memory");
     }
-#undef HS_META
-    if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
-    if (fast) {
-      // nothing to fetch: let whatever follows in the stream start its prologue now (measured: with a fetch ahead,
-      // releasing the dependents before the first loads are issued costs the fetch about 2 us, so that path
-      // releases them only once its metadata is written back)
-      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-      // Every valid selection is resident (or the newest record): the slot table, the hit stamps in slot order
-      // (coalesced) and the counters are all there is to write.  The recency list is not touched and
-      // order_t stays behind; under FIFO a hit changes nothing, so the list stays current.
-      int32_t *trow = table + (int64_t)r * k;
-      int32_t *arow = d.anchor_out + rg * k;
-      for (int j = tid; j < k; j += T) {
-        const int32_t o = s_out[j];
-        trow[j] = o < 0 ? -1 : r * (B + 1) + o;
-        if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
-      }
-      int c = 0;
-      for (int w = tid; w < W; w += T) c += __popc(s_hitbits[w]);
-      if (warp * 32 < W) {
-        c = __reduce_add_sync(0xffffffffu, c);
-        if (lane == 0 && c) atomicAdd(&s_misc[3], c);
-      }
-      if (d.policy != HISPARSE_POLICY_FIFO) {
-        uint32_t *last_use = d.last_use + rg * B;
-        for (int s = tid; s < B; s += T)
-          if ((s_hitbits[s >> 5] >> (s & 31)) & 1u) last_use[s] = 2u * t + 1u;
-      }
-      __syncthreads();
-      if (tid == 0) {
-        const int nhits = s_misc[3] + (s_misc[2] ? 1 : 0);
-        hits_out[r] = nhits;
-        misses_out[r] = 0;
-        d.anchor_hits[rg] = nhits;
-        d.anchor_misses[rg] = 0;
-        d.plan_n[rg] = 0;
-        d.t[rg] = t;
-        if (d.policy == HISPARSE_POLICY_FIFO) d.order_t[rg] = t;
-        if (timers) stamps[4] = global_ns();
-      }
-    } else {
-      // Phase 4 starts here, with the positions of the misses: the first batch of host loads is in flight while the
-      // victims are chosen (a record's slot is only needed when it is stored) and the metadata is written back
-      fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
-      fetch.issue(d);
-#define HS_VICT(IPT)                                                                                              \
-  choose_victims<T, IPT>(d, r, rg, m, s_plan_slot, s_tab, s_hitbits, s_vicbits, s_order, s_warp, s_vicpre, stamps, t, \
-                         order_t, n_nonhit)
-      if constexpr (T == kThreads) {
-        if (B <= 4 * T) HS_VICT(4);
-        else if (B <= 8 * T) HS_VICT(8);
-        else HS_VICT(16);
-      } else {
-        if (B <= 8 * T) HS_VICT(8);
-        else HS_VICT(16);
-      }
+  } else {
+    stage_async(v.order, order_g, B * 2);
+  }
+  list_misses<T, KPT>(d, v, c.trow, c.arow, stamps, s_misc, pos, cls, my_status, m);
+  if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
+  // Phase 4 starts here, with the positions of the misses: the first batch of host loads is in flight while the
+  // victims are chosen (a record's slot is only needed when it is stored) and the metadata is written back
+  TmaFetch fetch;
+  fetch.init(d, r, c.layer, m, v.plan_pos, v.plan_slot, v.ring, v.bars, 0, S, fetch_parity);
+  fetch.issue(d);
+#define HS_VICT(IPT) choose_victims<T, IPT>(d, v, r, rg, m, stamps, t, order_t, order_bulk, order_parity, my_status, n_nonhit)
+  if constexpr (T == kThreads) {
+    if (B <= 4 * T) HS_VICT(4);
+    else if (B <= 8 * T) HS_VICT(8);
+    else HS_VICT(16);
+  } else {
+    if (B <= 8 * T) HS_VICT(8);
+    else HS_VICT(16);
+  }
 #undef HS_VICT
-      // same state as right after the first issue, recomputed instead of kept in registers across the victim choice
-      fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, 0, S);
-      fetch.active = fetch.active && fetch.piece_of(d, 0) < fetch.total;
-      // Phase 5, metadata half: page table, slot array, stamps, plan
-      int32_t *slot_pos = d.slot_pos + rg * B;
-      uint32_t *last_use = d.last_use + rg * B;
-      int16_t *p2s = d.pos2slot + p2s_off_r + (int64_t)g * cap_r;
-      int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
-      for (int i = tid; i < m; i += T) {
-        const int v = s_plan_slot[i];
-        const int32_t p = s_plan_pos[i];
-        const int32_t old = slot_pos[v];
-        if (old >= 0) p2s[old] = -1;
-        slot_pos[v] = p;
-        p2s[p] = (int16_t)v;
-        last_use[v] = miss_stamp;
-        plan_pos_g[i] = p;
-        plan_slot_g[i] = v;
-      }
-      if (tid == 0) d.plan_n[rg] = m;
+  if (order_bulk) order_parity ^= 1u;
+  // same state as right after the first issue, recomputed instead of kept in registers across the victim choice
+  fetch.init(d, r, c.layer, m, v.plan_pos, v.plan_slot, v.ring, v.bars, 0, S, fetch_parity);
+  fetch.active = fetch.active && fetch.piece_of(d, 0) < fetch.total;
+  // Phase 5, metadata half: page table, slot array, stamps, plan, and the slot-table entries of the misses
+  {
+    int32_t *slot_pos = d.slot_pos + rg * B;
+    uint32_t *last_use = d.last_use + rg * B;
+    int16_t *p2s = d.pos2slot + c.p2s_off_r + (int64_t)c.g * p2s_stride(c.cap_r);
+    int32_t *plan_pos_g = d.plan_pos + rg * k, *plan_slot_g = d.plan_slot + rg * k;
+    const int32_t base = r * (B + 1);
+    const uint32_t miss_stamp = 2u * t;
+    for (int i = tid; i < m; i += T) {
+      const int vs = v.plan_slot[i];
+      const int32_t p = v.plan_pos[i];
+      const int j = v.missj[i];
+      const int32_t old = slot_pos[vs];
+      if (old >= 0) p2s[old] = -1;
+      slot_pos[vs] = p;
+      p2s[p] = (int16_t)vs;
+      last_use[vs] = miss_stamp;
+      plan_pos_g[i] = p;
+      plan_slot_g[i] = vs;
+      c.trow[j] = base + vs;
+      if (c.arow) c.arow[j] = vs;
     }
-    if (my_status) atomicOr(d.status, my_status);
+    if (tid == 0) d.plan_n[rg] = m;
   }
+  if (my_status) atomicOr(d.status, my_status);
+  if (my_status & HISPARSE_STATUS_TIMEOUT) gave_up = true;
   // The plan is public: the other blocks of the cluster start fetching while this one publishes.  Every thread
   // arrives with release semantics after its own plan writes and every reader waits with acquire semantics, which
   // orders them at cluster scope: no separate fence.
-  if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-
-  if (part == 0 && !fast) {
+  if (S > 1) cluster_arrive();
+  {
     uint16_t *order = d.order + rg * B;
+    uint32_t *s_hitbits = v.hitbits, *s_vicbits = v.vicbits;
+    int32_t *s_hitpre = v.hitpre, *s_vicpre = v.vicpre;
+    uint16_t *s_order = v.order;
     // new order = untouched ++ victims by slot ++ hits by slot: word-level prefix counts, then one pass.
     if (warp == 0) {
       int run_h = 0, run_v = 0;
@@ -775,17 +832,18 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
         run_v += __shfl_sync(0xffffffffu, iv, 31);
       }
     }
-    // Phase 5: the slot table in selection order (does not depend on the order rewrite)
-    int32_t *trow = table + (int64_t)r * k;
-    int32_t *arow = d.anchor_out + rg * k;
-    for (int j = tid; j < k; j += T) {
-      int32_t o = s_out[j];
-      if (o <= kDupBase && o > kRankBase) o = s_out[kDupBase - o];  // a repeated position follows its first occurrence
-      if (o <= kRankBase) o = s_plan_slot[kRankBase - o];           // a miss takes its victim's slot
-      trow[j] = o < 0 ? -1 : r * (B + 1) + o;
-      if (d.lpg > 1) arow[j] = o < 0 ? -1 : o;
-    }
     __syncthreads();
+    if (s_misc[0]) {
+      // rare: a row entry that repeats a missing position takes the table entry of its first occurrence, which this
+      // block wrote above (block-scope ordering through the barrier)
+      for (int j = tid; j < k; j += T) {
+        const int32_t o = c.trow[j];
+        if (o <= kDupBase) {
+          c.trow[j] = c.trow[kDupBase - o];
+          if (c.arow) c.arow[j] = c.arow[kDupBase - o];
+        }
+      }
+    }
     uint32_t *last_use = d.last_use + rg * B;
     if (d.policy == HISPARSE_POLICY_FIFO) {
       // insertion order: the refilled slots go to the end, by slot; hits were left where they were, unstamped
@@ -809,12 +867,15 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
       }
     }
     __syncthreads();
-    for (int q = tid; q < B; q += T) order[q] = s_order[q];
+    for (int qq = tid; qq < B; qq += T) order[qq] = s_order[qq];
     if (tid == 0) {
-      // distinct hits = slots whose hit bit is set (+ the reserved slot if the newest position was selected)
+      // distinct hits = slots whose hit bit is set (+ the reserved slot if the newest position was selected); more
+      // selections that hit than slots hit = a resident position was selected twice
       const int nhits = (B - n_nonhit) + (s_misc[2] ? 1 : 0);
-      hits_out[r] = nhits;
-      misses_out[r] = m;
+      if (s_misc[1] != B - n_nonhit) atomicOr(d.status, HISPARSE_STATUS_DUPLICATE);
+      s_misc[0] = s_misc[1] = s_misc[2] = s_misc[3] = 0;  // this set serves the request after the next
+      c.hits_out[r] = nhits;
+      c.misses_out[r] = m;
       d.anchor_hits[rg] = nhits;
       d.anchor_misses[rg] = m;
       d.t[rg] = t;
@@ -822,28 +883,486 @@ resolve_kernel(const DevState d, const int layer, const int32_t *__restrict__ se
     }
     if (timers && tid == 0) stamps[4] = global_ns();
   }
-
-  if (S > 1) {
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    if (part != 0) {
-      m = __ldcg(d.plan_n + rg);
-      const int32_t *pp = d.plan_pos + rg * k, *ps = d.plan_slot + rg * k;
-      for (int i = tid; i < m; i += T) { s_plan_pos[i] = __ldcg(pp + i); s_plan_slot[i] = __ldcg(ps + i); }
-      __syncthreads();
-      fetch.init(d, r, layer, m, s_plan_pos, s_plan_slot, s_ring, s_bars, part, S);
-      fetch.issue(d);
-    }
-  }
+  if (S > 1) cluster_wait();
   // Phase 4, rest: wait for the batches, store them into the cache slots, issue what is left.  Whatever follows
   // in the stream may be scheduled from here on (it still waits for this grid to finish before it reads).
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  fetch.drain(d, d.status);
+  if (!c.has_next) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!fetch.drain(d, d.status)) gave_up = true;
+  fetch_parity = fetch.parity;
   if (timers) {
     __syncthreads();
     if (tid == 0) {
       const unsigned long long now = global_ns();
-      if (part == 0) stamps[5] = now;
+      stamps[5] = now;
       atomicMax(&stamps[6], now);
+    }
+  }
+}
+
+// The same, kept out of line for blocks that loop over requests: the loop's short path (nothing missed) then keeps
+// its few registers, and only a request with misses pays for the call.  The thread's row entries and their
+// classification travel through shared memory (the victim array is idle until the victims are chosen).
+template <int T, int KPT>
+__device__ __noinline__ void miss_path_cold(const DevState &d, const ReqCtx &c, const uint32_t t, const uint32_t order_t,
+                                            const uint32_t my_status, uint32_t &fetch_parity, uint32_t &order_parity,
+                                            bool &gave_up) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  static_assert(KPT == 4, "the stash holds one position per row entry");
+  int32_t pos[KPT], cls[KPT];
+  int4 x = make_int4(-1, -1, -1, -1);
+  if ((int)threadIdx.x * KPT < d.k) x = reinterpret_cast<const int4 *>(smem_raw + d.sm_plan_slot)[threadIdx.x];
+  pos[0] = x.x; pos[1] = x.y; pos[2] = x.z; pos[3] = x.w;
+#pragma unroll
+  for (int i = 0; i < KPT; ++i) cls[i] = pos[i] >= 0 ? kMiss : -1;  // only the misses matter from here on
+  // (the array gets its real content only after several block barriers: every thread has its entries by then)
+  miss_path<T, KPT>(d, c, pos, cls, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+}
+
+// A block of a cluster other than the first: shares the page-table lookups when the slice cannot be staged, then
+// takes its share of the recorded plan through the fetch pipeline.
+template <int T>
+__device__ __forceinline__ void helper_block(const DevState &d, const ReqCtx &c, const int part, uint32_t &fetch_parity,
+                                             bool &gave_up) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const SmemView v = smem_view(d, smem_raw, 0);
+  const int tid = threadIdx.x, k = d.k;
+  const SliceGeom q = slice_geom(d, c.g, c.cap_r, c.p2s_off_r);
+  if (!q.staged) {  // the request's page-table slice is too large to be staged: the cluster shares the lookups
+    const int64_t na = *(volatile int32_t *)d.n_appends;
+    const int64_t len = c.init_len_r + na < c.cap_r ? c.init_len_r + na : c.cap_r;
+    cluster_arrive_relaxed();  // phase A
+    cluster_lookups<T>(c.row, q.p2s, k, len, part, c.S, v.got);
+  }
+  cluster_arrive();
+  cluster_wait();
+  const int m = __ldcg(d.plan_n + c.rg);
+  const int32_t *pp = d.plan_pos + c.rg * k, *ps = d.plan_slot + c.rg * k;
+  for (int i = tid; i < m; i += T) { v.plan_pos[i] = __ldcg(pp + i); v.plan_slot[i] = __ldcg(ps + i); }
+  __syncthreads();
+  TmaFetch fetch;
+  fetch.init(d, c.r, c.layer, m, v.plan_pos, v.plan_slot, v.ring, v.bars, part, c.S, fetch_parity);
+  fetch.issue(d);
+  if (!fetch.drain(d, d.status)) gave_up = true;
+  fetch_parity = fetch.parity;
+  if (d.flags & HISPARSE_FLAG_PHASE_TIMERS) {
+    __syncthreads();
+    if (tid == 0) atomicMax(&d.phase_ns[(int64_t)c.r * 16 + 6], global_ns());
+  }
+}
+
+// The loop of a resident wave of narrow blocks, written out for the shape it is meant for: every request has the
+// same capacity, the rows / table rows / page-table slices are 16-byte aligned whole units, the slice fits the ring.
+// Same steps and same results as the general code below (lookup_phase + the short path of resolve_kernel), with
+// everything that does not depend on the request hoisted out of the loop, 32-bit lengths, and no per-request geometry
+// structs: the general code spends ~840 instructions per thread and request, which made a resolve in which nothing
+// misses issue-bound; this loop spends about a fifth of that.  A request with a miss leaves through miss_path_cold.
+__device__ __forceinline__ bool lean_shape(const DevState &d, const int32_t *sel, const int32_t *table, const int threads) {
+  return !(d.flags & HISPARSE_FLAG_PHASE_TIMERS) && d.uni_cap >= 0 && d.order_t != nullptr &&
+         (((uintptr_t)sel | (uintptr_t)table | (uintptr_t)d.pos2slot | (uintptr_t)d.anchor_out) & 15) == 0 &&
+         (d.k & 3) == 0 && d.k <= 4 * threads && p2s_stride(d.uni_cap) * 2 + 16 <= (int64_t)d.ring_bytes;
+}
+
+template <int T>
+__device__ __forceinline__ void lean_stage_issue(const DevState &d, const int32_t *sel, const int g, const int r,
+                                                 const uint32_t s_sel_addr, const uint32_t ring_addr, const uint32_t stage_bar) {
+  const uint32_t lane = threadIdx.x;  // called by the first warp only
+  const uint32_t row_bytes = (uint32_t)d.k * 4u;
+  const uint32_t slice_bytes = (uint32_t)p2s_stride(d.uni_cap) * 2u;  // whole 16-byte units (the padding is -1)
+  if (lane == 0)
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(stage_bar), "r"(row_bytes + slice_bytes) : "memory");
+  const char *row = reinterpret_cast<const char *>(sel + (int64_t)r * d.k);
+  const char *slice = reinterpret_cast<const char *>(d.pos2slot + ((int64_t)r * d.G + g) * p2s_stride(d.uni_cap));
+  const uint32_t row_pieces = (row_bytes + kStagePiece - 1) / kStagePiece, slice_pieces = (slice_bytes + kStagePiece - 1) / kStagePiece;
+  for (uint32_t p = lane; p < row_pieces + slice_pieces; p += 32u) {  // small pieces, side by side: see stage_issue
+    const bool in_row = p < row_pieces;
+    const uint32_t o = (in_row ? p : p - row_pieces) * kStagePiece, total = in_row ? row_bytes : slice_bytes;
+    const uint32_t n = total - o < kStagePiece ? total - o : kStagePiece;
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"((in_row ? s_sel_addr : ring_addr) + o), "l"((in_row ? row : slice) + o), "r"(n), "r"(stage_bar) : "memory");
+  }
+}
+
+// Shared-memory accesses of the lean loop by 32-bit shared address (no generic-address arithmetic).
+__device__ __forceinline__ int4 lds_v4(uint32_t a) {
+  int4 v;
+  asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ int32_t lds_s16(uint32_t a) {
+  int32_t v;
+  asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_u8(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts_u8(uint32_t a, uint32_t v) { asm volatile("st.shared.u8 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ int32_t lds_s32(uint32_t a) {
+  int32_t v;
+  asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_s32(uint32_t a, int32_t v) { asm volatile("st.shared.s32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ void red_add_s32(uint32_t a, int32_t v) { asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ int32_t atom_add_s32(uint32_t a, int32_t v) {
+  int32_t o;
+  asm volatile("atom.shared.add.s32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
+  return o;
+}
+
+// What miss_path_cold hands back to a looping block, packed into one word (no locals whose address is taken).
+constexpr uint32_t kColdFetchParity = 1u, kColdOrderParity = 2u, kColdGaveUp = 4u;
+
+template <int T>
+__device__ __noinline__ uint32_t lean_miss(const DevState &d, const int layer, const int g, const int32_t *sel, int32_t *table,
+                                           int32_t *hits_out, int32_t *misses_out, const int r, const int it, const int tag,
+                                           const bool has_next, const uint32_t t, const uint32_t st, const uint32_t state) {
+  const int k = d.k;
+  const int64_t cap = d.uni_cap;
+  ReqCtx c;
+  c.r = r; c.it = it; c.S = 1; c.layer = layer; c.g = g; c.rg = (int64_t)r * d.G + g;
+  c.cap_r = cap; c.init_len_r = d.uni_init_len; c.p2s_off_r = (int64_t)r * d.G * p2s_stride(cap);
+  c.row = sel + (int64_t)r * k;
+  c.trow = table + (int64_t)r * k;
+  c.arow = d.lpg > 1 ? d.anchor_out + c.rg * k : nullptr;
+  c.hits_out = hits_out; c.misses_out = misses_out;
+  c.has_next = has_next; c.tag = tag;
+  uint32_t fetch_parity = state & kColdFetchParity, order_parity = (state & kColdOrderParity) ? 1u : 0u;
+  bool gave_up = false;
+  miss_path_cold<T, 4>(d, c, t, d.order_t[c.rg], st, fetch_parity, order_parity, gave_up);
+  return fetch_parity | (order_parity ? kColdOrderParity : 0u) | (gave_up ? kColdGaveUp : 0u);
+}
+
+template <int T>
+__device__ __forceinline__ void lean_loop(const DevState &d, const int layer, const int g, const int32_t *__restrict__ sel,
+                                          int32_t *__restrict__ table, int32_t *__restrict__ hits_out,
+                                          int32_t *__restrict__ misses_out, int r, const int stride) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int k = d.k, B = d.B, N = d.N;
+  const uint32_t a_base = smem_u32(smem_raw);
+  const uint32_t a_ring = a_base + (uint32_t)(d.meta_smem + d.bar_bytes);   // the staged page-table slice
+  const uint32_t a_marks = a_base + (uint32_t)d.sm_marks;
+  const uint32_t a_spare = a_marks + (uint32_t)d.marks_spare;                // a byte that no slot owns
+  const uint32_t a_misc = a_base + (uint32_t)d.sm_misc + 128u;              // two sets of 8 ints
+  const uint32_t a_stash = a_base + (uint32_t)d.sm_plan_slot + (uint32_t)tid * 16u;
+  const uint32_t stage_bar = a_base + (uint32_t)d.meta_smem + (uint32_t)T * 8u;
+  const uint32_t a_row = a_base + (uint32_t)tid * 16u;                      // this thread's four row entries
+  const int cap = (int)d.uni_cap, il = (int)d.uni_init_len;
+  const bool mine = tid * 4 < k;
+  const bool stamp_hits = d.policy != HISPARSE_POLICY_FIFO;
+  const int G = d.G;
+  uint32_t state = 0;   // kCold* bits: phases of the fetch / list barriers as the out-of-line path left them
+  int tag = 0;
+  uint32_t parity = 0;
+  // nothing appends while a resolve runs (stream order): the lengths are the same for every request of the launch
+  const int na = *(volatile int32_t *)d.n_appends;
+  int len = il + na, newest = na > 0 ? il + na - 1 : -2;  // -2: no newest record (a discarded entry is -1)
+  if (len > cap) { len = cap; newest = -2; }
+  // a request's resolve count is loaded one request ahead (with the next request's inputs), so that the trip to
+  // memory is over when the count is needed
+  uint32_t t_ahead = r < N ? d.t[r * G + g] : 0u;
+  for (; r < N; r += stride, parity ^= 1u) {
+    const int rg = r * G + g;                       // N * G fits 32 bits (the metadata arrays are indexed by it)
+    const uint32_t a_set = a_misc + parity * 32u;
+    if (tag == 255) {
+      // the tags start over: forget the old marks (every thread is done with the previous request's)
+      tag = 0;
+      for (int i = tid * 16; i < B; i += T * 16) *reinterpret_cast<uint4 *>(smem_raw + d.sm_marks + i) = make_uint4(0, 0, 0, 0);
+      __syncthreads();
+    }
+    ++tag;
+    const uint32_t t = t_ahead + 1u;
+    bool landed = true;
+    if (tid < 32 && !mbar_wait_bounded(stage_bar, parity)) {
+      mbar_wait_bounded(stage_bar, parity);
+      landed = false;
+    }
+    uint32_t st = 0;
+    bool gave_up = false;
+    if (__syncthreads_or(!landed)) { st = HISPARSE_STATUS_TIMEOUT; gave_up = true; }
+    int4 x = make_int4(-1, -1, -1, -1);
+    if (mine && !gave_up) x = lds_v4(a_row);
+    int32_t pos[4] = {x.x, x.y, x.z, x.w};
+    int32_t got[4];
+    int bad = 0;
+    // every access below is unconditional (an entry that is padding or out of range looks up position 0 and discards
+    // the answer; an entry that did not hit marks a spare byte): branches around them cost more than they save
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const bool ok = (uint32_t)pos[i] < (uint32_t)len;  // 0 <= p < len
+      bad |= (!ok) & (pos[i] != -1);
+      const int32_t g16 = lds_s16(a_ring + 2u * (uint32_t)(ok ? pos[i] : 0));
+      pos[i] = ok ? pos[i] : -1;
+      got[i] = ok ? g16 : -1;
+    }
+    if (bad) st |= HISPARSE_STATUS_OUT_OF_RANGE;
+    const int32_t base = r * (B + 1);
+    int nhit = 0, nnew = 0;
+    bool miss = false;
+    int32_t val[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      // (the newest position is never resident in an LRU slot: its record sits in the reserved slot)
+      const bool isnew = pos[i] == newest, hit = got[i] >= 0;
+      miss |= pos[i] >= 0 && !isnew && !hit;
+      sts_u8(hit ? a_marks + (uint32_t)got[i] : a_spare, (uint32_t)tag);
+      nhit += hit;
+      nnew += isnew;
+      val[i] = hit ? base + got[i] : (isnew ? base + B : -1);
+    }
+    if (nnew) {  // the reserved newest-record slot, outside the LRU set; selected twice = a repeated position
+      if (atom_add_s32(a_set + 8u, nnew) + nnew > 1) st |= HISPARSE_STATUS_DUPLICATE;
+    }
+    if (mine) {
+      *reinterpret_cast<int4 *>(table + (int64_t)r * k + tid * 4) = make_int4(val[0], val[1], val[2], val[3]);
+      if (d.lpg > 1)
+        *reinterpret_cast<int4 *>(d.anchor_out + (int64_t)rg * k + tid * 4) =
+            make_int4(val[0] < 0 ? -1 : val[0] - base, val[1] < 0 ? -1 : val[1] - base, val[2] < 0 ? -1 : val[2] - base,
+                      val[3] < 0 ? -1 : val[3] - base);
+    }
+    nhit = __reduce_add_sync(0xffffffffu, nhit);
+    if (lane == 0 && nhit) red_add_s32(a_set + 4u, nhit);
+    const bool has_next = r + stride < N;
+    if (has_next) t_ahead = d.t[rg + stride * G];
+    if (__syncthreads_or(miss)) {
+      // something missed: the general path, out of line; the thread's missing positions travel through shared memory
+      if (mine) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sts_s32(a_stash + 4u * i, (pos[i] >= 0 && pos[i] != newest && got[i] < 0) ? pos[i] : -1);
+      }
+      state = lean_miss<T>(d, layer, g, sel, table, hits_out, misses_out, r, (int)parity, tag, has_next, t, st, state);
+      if (has_next) {  // after a fetch, the next request's inputs can only start once every thread is done with the ring
+        if (__syncthreads_or((state & kColdGaveUp) != 0)) return;
+        if (tid < 32) lean_stage_issue<T>(d, sel, g, r + stride, a_base, a_ring, stage_bar);
+      }
+      continue;
+    }
+    if (has_next && !gave_up) {
+      // the row and the ring are free (every thread consumed its entries before the vote): the next request's inputs
+      // travel while this one's stamps are written
+      if (tid < 32) lean_stage_issue<T>(d, sel, g, r + stride, a_base, a_ring, stage_bar);
+    } else {
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+    {
+      uint32_t *lu = d.last_use + (int64_t)rg * B + tid;
+      const uint32_t hit_stamp = 2u * t + 1u;
+      const uint32_t a_m = a_marks + (uint32_t)tid;
+      int cnt = 0;
+      for (int s0 = 0; s0 < B; s0 += 4 * T) {   // the marks are padded to whole rounds of this loop (padding = 0)
+        uint32_t m[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m[j] = lds_u8(a_m + (uint32_t)(s0 + j * T));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const bool hit = m[j] == (uint32_t)tag;
+          if (hit && stamp_hits) lu[s0 + j * T] = hit_stamp;
+          cnt += hit;
+        }
+      }
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if (lane == 0 && cnt) red_add_s32(a_set + 12u, cnt);
+    }
+    __syncthreads();  // the counts are complete, and the marks may be written again
+    if (tid == 0) {
+      const int distinct = lds_s32(a_set + 12u), selected = lds_s32(a_set + 4u), isnew = lds_s32(a_set + 8u);
+      if (distinct != selected) st |= HISPARSE_STATUS_DUPLICATE;  // a resident position was selected twice
+      const int nhits = distinct + (isnew ? 1 : 0);
+      sts_s32(a_set, 0); sts_s32(a_set + 4u, 0); sts_s32(a_set + 8u, 0); sts_s32(a_set + 12u, 0);  // for the request after the next
+      hits_out[r] = nhits;
+      misses_out[r] = 0;
+      d.anchor_hits[rg] = nhits;
+      d.anchor_misses[rg] = 0;
+      d.plan_n[rg] = 0;
+      d.t[rg] = t;
+      if (!stamp_hits) d.order_t[rg] = t;
+    }
+    if (st) atomicOr(d.status, st);
+    if (gave_up) return;
+  }
+}
+
+// MINB = thread blocks of this size that must fit one SM (bounds the registers per thread).
+// Grid: one cluster of S blocks per request, or fewer clusters than requests, in which case a cluster takes the
+// requests c, c + clusters, c + 2 clusters, .. one after the other (LOOP, only with S = 1: a grid of several waves is
+// launched as one resident wave of looping blocks, so that no block pays for another launch and the next request's
+// row and page-table slice are already on their way while the current one is finished).
+template <int T, int MINB, bool LOOP>
+__global__ void __launch_bounds__(T, MINB)
+resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_t *__restrict__ sel,
+               int32_t *__restrict__ table, int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out, const int S) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int part = blockIdx.x % S, stride = gridDim.x / S;
+  const int g = layer / d.lpg;
+  const int k = d.k, B = d.B, W = d.W;
+  const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
+
+  // Prologue that depends on nothing an earlier kernel wrote: barriers, cleared marks (and table, when it has memory
+  // of its own), the addresses of everything Phase 1 will load.  With programmatic dependent launch it overlaps the
+  // tail of whatever runs before this kernel in the stream.
+  int r = blockIdx.x / S;
+  {
+    const SmemView v = smem_view(d, smem_raw, 0);
+    fetch_barriers_init(v.bars, d.io_threads);
+    if (part == 0) {
+      if (d.sm_tab >= 0)
+        for (int i = tid; i < d.H; i += T) v.tab[i] = kEmptyEntry;
+      for (int i = tid * 16; i < d.marks_spare + 16; i += T * 16) *reinterpret_cast<uint4 *>(v.marks + i) = make_uint4(0, 0, 0, 0);
+      if (tid < 16) v.misc[tid] = 0;
+      if (tid < 2) {
+        // Warm L2 with what Phase 1 will stage (row, page-table slice).  A prefetch consumes nothing, and L2 is where
+        // earlier kernels' writes land, so this is safe before the dependency wait; when the previous kernel lets its
+        // dependents start early, the staging after the wait then reads L2 instead of HBM.
+        int64_t cap_r, init_len_r, p2s_off_r;
+        request_geom(d, r, cap_r, init_len_r, p2s_off_r);
+        const SliceGeom q = slice_geom(d, g, cap_r, p2s_off_r);
+        const char *p = tid == 0 ? reinterpret_cast<const char *>(sel + (int64_t)r * k) : reinterpret_cast<const char *>(q.p2s);
+        int64_t n = tid == 0 ? (int64_t)k * 4 : cap_r * 2;
+        const uintptr_t a = ((uintptr_t)p + 15) & ~(uintptr_t)15;   // whole 16-byte units inside the array only
+        n = (n - (int64_t)(a - (uintptr_t)p)) & ~(int64_t)15;
+        if (n > (1 << 20)) n = 1 << 20;                             // no point warming more than the ring could stage
+        if (n > 0 && (tid == 0 || q.staged))
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a), "r"((uint32_t)n) : "memory");
+      }
+    }
+    __syncthreads();  // the barriers are initialised and the marks cleared before anything uses them
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (part != 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (part == 0) {
+      int64_t cap_r, init_len_r, p2s_off_r;
+      request_geom(d, r, cap_r, init_len_r, p2s_off_r);
+      stage_issue<T>(d, v, slice_geom(d, g, cap_r, p2s_off_r), sel + (int64_t)r * k, cap_r, smem_u32(v.bars + T));
+    }
+  }
+  uint32_t fetch_parity = 0, order_parity = 0;  // phases of this thread's fetch barrier / of the list's staging barrier
+  bool gave_up = false;                          // a bounded wait expired: the block takes no further request
+
+  if constexpr (LOOP) {
+    if (S == 1 && lean_shape(d, sel, table, T)) {
+      lean_loop<T>(d, layer, g, sel, table, hits_out, misses_out, r, stride);
+      return;
+    }
+  }
+  // (the wide block never loops: one pass, so that nothing has to stay in registers across requests)
+  for (int it = 0; r < d.N && !gave_up && (LOOP || it == 0); r += stride, ++it) {
+    ReqCtx c;
+    c.r = r; c.it = it; c.S = S; c.layer = layer; c.g = g;
+    c.rg = (int64_t)r * d.G + g;
+    request_geom(d, r, c.cap_r, c.init_len_r, c.p2s_off_r);
+    c.row = sel + (int64_t)r * k;
+    c.trow = table + (int64_t)r * k;
+    c.arow = d.lpg > 1 ? d.anchor_out + c.rg * k : nullptr;
+    c.hits_out = hits_out; c.misses_out = misses_out;
+    c.has_next = LOOP && r + stride < d.N;
+    if (part != 0) {
+      helper_block<T>(d, c, part, fetch_parity, gave_up);
+      continue;
+    }
+    const SmemView v = smem_view(d, smem_raw, it);
+    const SliceGeom q = slice_geom(d, g, c.cap_r, c.p2s_off_r);
+    unsigned long long *stamps = d.phase_ns + (int64_t)r * 16;
+    if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
+    c.tag = it % 255 + 1;
+    if (LOOP && it > 0 && c.tag == 1) {
+      // the tags start over: forget the old marks (every thread is done with the previous request's)
+      for (int i = tid * 16; i < B; i += T * 16) *reinterpret_cast<uint4 *>(v.marks + i) = make_uint4(0, 0, 0, 0);
+      __syncthreads();
+    }
+    uint32_t my_status = 0, order_t = 0, t = 0;
+    bool any_miss = false;
+    // row entries per thread: k <= 4 * T by construction (create refuses other shapes for this block size)
+    constexpr int KPT = 4;
+    int32_t pos[KPT], cls[KPT];
+    if (!LOOP && k <= 2 * T) {
+      int32_t pos2[2], cls2[2];
+      lookup_phase<T, 2>(d, v, q, c, (uint32_t)(it & 1), stamps, pos2, cls2, my_status, any_miss, t, order_t);
+      if (any_miss || d.order_t == nullptr) {
+        miss_path<T, 2>(d, c, pos2, cls2, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+        continue;
+      }
+    } else {
+      lookup_phase<T, KPT>(d, v, q, c, (uint32_t)(it & 1), stamps, pos, cls, my_status, any_miss, t, order_t);
+      if (any_miss || d.order_t == nullptr) {
+        if (LOOP) {
+          // stash the thread's missing positions for the out-of-line path
+          if (tid * KPT < k)
+            reinterpret_cast<int4 *>(v.plan_slot)[tid] = make_int4(cls[0] == kMiss ? pos[0] : -1, cls[1] == kMiss ? pos[1] : -1,
+                                                                  cls[2] == kMiss ? pos[2] : -1, cls[3] == kMiss ? pos[3] : -1);
+          const ReqCtx cc = c;  // the copy that lives in memory for the call; `c` itself stays in registers
+          miss_path_cold<T, KPT>(d, cc, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+          if (c.has_next) {
+            // after a fetch, the next request's inputs can only start once every thread is done with the ring
+            gave_up = __syncthreads_or(gave_up) != 0;
+            if (!gave_up) {
+              const int rn = r + stride;
+              int64_t cap_n, il_n, off_n;
+              request_geom(d, rn, cap_n, il_n, off_n);
+              stage_issue<T>(d, v, slice_geom(d, g, cap_n, off_n), sel + (int64_t)rn * k, cap_n, smem_u32(v.bars + T));
+            }
+          }
+        } else {
+          miss_path<T, KPT>(d, c, pos, cls, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+        }
+        continue;
+      }
+    }
+    // Short path.  Every valid selection is resident (or the newest record): nothing to fetch, no victim to choose.
+    // The slot table is written; what is left are the hit stamps, in slot order (coalesced), and the counters.  The
+    // recency list is not touched and order_t stays behind (rebuild_order brings it up to date in the next resolve
+    // that needs victims); under FIFO a hit changes nothing, so the list stays current.
+    if (my_status & HISPARSE_STATUS_TIMEOUT) gave_up = true;
+    if (c.has_next && !gave_up) {
+      // the row and the ring are free (every thread consumed its entries before the vote): the next request's
+      // inputs travel while this one's stamps are written
+      const int rn = r + stride;
+      int64_t cap_n, il_n, off_n;
+      request_geom(d, rn, cap_n, il_n, off_n);
+      stage_issue<T>(d, v, slice_geom(d, g, cap_n, off_n), sel + (int64_t)rn * k, cap_n, smem_u32(v.bars + T));
+    } else {
+      // let whatever follows in the stream start its prologue now (measured: with a fetch ahead, releasing the
+      // dependents before the first loads are issued costs the fetch about 2 us, so that path releases them only
+      // once its metadata is written back)
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+    if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
+    {
+      uint32_t *last_use = d.last_use + c.rg * B;
+      const uint32_t hit_stamp = 2u * t + 1u;
+      const bool stamp = d.policy != HISPARSE_POLICY_FIFO;
+      const uint8_t tag = (uint8_t)c.tag;
+      int cnt = 0;
+      for (int s = tid; s < B; s += T)
+        if (v.marks[s] == tag) {
+          if (stamp) last_use[s] = hit_stamp;
+          ++cnt;
+        }
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if (lane == 0 && cnt) atomicAdd(&v.misc[3], cnt);
+    }
+    // the counts are complete, and the marks may be written again (a looping block's next request)
+    __syncthreads();
+    if (tid == 0) {
+      const int distinct = v.misc[3];
+      if (distinct != v.misc[1]) my_status |= HISPARSE_STATUS_DUPLICATE;  // a resident position was selected twice
+      const int nhits = distinct + (v.misc[2] ? 1 : 0);
+      v.misc[0] = v.misc[1] = v.misc[2] = v.misc[3] = 0;  // this set serves the request after the next
+      hits_out[r] = nhits;
+      misses_out[r] = 0;
+      d.anchor_hits[c.rg] = nhits;
+      d.anchor_misses[c.rg] = 0;
+      d.plan_n[c.rg] = 0;
+      d.t[c.rg] = t;
+      if (d.policy == HISPARSE_POLICY_FIFO) d.order_t[c.rg] = t;
+      if (timers) stamps[4] = global_ns();
+    }
+    if (my_status) atomicOr(d.status, my_status);
+    if (S > 1) {  // the other blocks of the cluster find an empty plan
+      cluster_arrive();
+      cluster_wait();
     }
   }
 }
