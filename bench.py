@@ -13,12 +13,16 @@ records, k = 2048, B = 4096, ~19.5 GB of pinned host history).
 Prints ONE JSON line (rank 0).  `value` = resolved selections per second over K timed steps with
 all inputs resident in HBM; `e2e` = the same through the public API with the step's inputs in pinned
 host memory (copied in inside the timed region) and the step's hit/miss counters read back.
+With --gpus N > 1 and no launcher in the environment the script starts N ranks of itself
+(torch.distributed.run on 127.0.0.1), one per GPU.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import re
+import socket
 import statistics
 import subprocess
 import sys
@@ -36,18 +40,19 @@ UNIT = "selections/s"
 ALGO_BYTES_PER_HIT = 16          # sel read + map probe + stamp write + slot-table write (4 B each)
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=24)
     ap.add_argument("--warmup", type=int, default=4)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "sharding-dry-run"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--overlap", type=float, default=0.9, help="c3 only: step-to-step selection overlap")
     ap.add_argument("--requests", type=int, default=0, help="override the number of requests (reduced runs)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (reduced runs)")
     ap.add_argument("--cache-slots", type=int, default=0, help="override B (cache-size sweeps)")
     ap.add_argument("--top-k", type=int, default=0, help="override k")
+    ap.add_argument("--context", type=int, default=0, help="override the history length (c2; tests)")
     ap.add_argument("--ctas-per-request", type=int, default=0)
     ap.add_argument("--no-prefetch", action="store_true", help="c3 only: shared layers swap in synchronously")
     ap.add_argument("--skip-io", action="store_true", help="no-IO timing mode (metadata only)")
@@ -55,27 +60,33 @@ def parse_args():
     ap.add_argument("--spec-hint", action="store_true",
                     help="speculative prefetch: layer l's selection is given to layer l+1 as a hint (side stream)")
     ap.add_argument("--no-pdl", action="store_true", help="launch Resolve without programmatic dependent launch")
-    ap.add_argument("--no-all-hit", action="store_true", help="skip the scaled all-hit HBM point")
+    ap.add_argument("--no-all-hit", action="store_true", help="skip the scaled all-hit HBM points")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--wide-blocks", action="store_true", help="1024-thread blocks even when the grid takes several waves")
     ap.add_argument("--eager-order", action="store_true", help="update the recency list in every resolve")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-requests", type=int, default=8)
     ap.add_argument("--cpu-sample-steps", type=int, default=200, help="oracle steps timed by the cpu_baseline leg")
-    return ap.parse_args()
+    return ap.parse_args(argv)
 
 
-def make_workload(args, rank: int = 0):
+def make_workload(args, rank: int = 0, name: str | None = None, steps: int | None = None):
+    """The workload a rank runs: configuration `name` (default: the one on the command line) with the command
+    line's overrides, seeded by the rank (weak scaling: every rank serves its own requests)."""
     from paper_2608_07009_b200 import inputs
-    steps = 2 * args.steps + args.warmup + 12         # cold + warm-up + timed + eager + e2e steps
-    seed = rank                      # weak scaling: every rank serves its own requests
-    if args.workload == "c1":
+    name = name or args.workload
+    if steps is None:
+        steps = 2 * args.steps + args.warmup + 12         # cold + warm-up + timed + eager + e2e steps
+    seed = rank
+    if name == "c1":
         w = inputs.c1_tiny_dsa(seed)
         w.steps = max(w.steps, steps)
-    elif args.workload == "c2":
-        w = inputs.c2_dsa_decode(seed, steps=steps)
-    elif args.workload == "c3":
+    elif name == "c2":
+        kw = dict(context=args.context) if args.context else {}
+        w = inputs.c2_dsa_decode(seed, steps=steps, **kw)
+    elif name == "c3":
         w = inputs.c3_dsa_long(args.overlap, seed, steps=steps)
-    elif args.workload == "c4":
+    elif name == "c4":
         w = inputs.c4_nsa_blocks(seed, steps=steps)
     else:
         w = inputs.c5_quest_pages(seed, steps=steps)
@@ -90,6 +101,66 @@ def make_workload(args, rank: int = 0):
         w.keep = round(w.keep * args.top_k / w.top_k)
         w.top_k = args.top_k
     return w
+
+
+# ----------------------------------------------------------------------------- launching N ranks
+
+
+def spawn_ranks(args, argv) -> int:
+    """`--gpus N` without a launcher in the environment: start N ranks of this script, one per GPU, and relay
+    rank 0's JSON line.  Refuses (non-zero exit) rather than silently running fewer ranks."""
+    import torch
+    if args.impl == "ours" and torch.cuda.device_count() < args.gpus:
+        print("bench.py: --gpus %d asked for, %d CUDA device(s) visible: not running a smaller job in its place"
+              % (args.gpus, torch.cuda.device_count()), file=sys.stderr)
+        return 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def gpu_numa_node(index: int):
+    """NUMA node of the PCIe root the GPU hangs off (None when the platform does not say)."""
+    try:
+        import torch
+        p = torch.cuda.get_device_properties(index)
+        bdf = "%04x:%02x:%02x.0" % (p.pci_domain_id, p.pci_bus_id, p.pci_device_id)
+        with open("/sys/bus/pci/devices/%s/numa_node" % bdf) as f:
+            node = int(f.read().strip())
+        return node if node >= 0 else None
+    except Exception:
+        return None
+
+
+def parse_cpulist(text: str):
+    cpus = set()
+    for part in text.strip().split(","):
+        if not part:
+            continue
+        lo, _, hi = part.partition("-")
+        cpus.update(range(int(lo), int(hi or lo) + 1))
+    return cpus
+
+
+def bind_near_gpu(index: int) -> dict:
+    """Runs this rank's threads on the CPUs of the GPU's NUMA node, so that the pinned histories it allocates next
+    (first touch) and the threads that fill them are local to the GPU's PCIe root.  Returns what was done."""
+    node = gpu_numa_node(index)
+    info = {"numa_node": node, "bound": False}
+    if node is None:
+        return info
+    try:
+        with open("/sys/devices/system/node/node%d/cpulist" % node) as f:
+            cpus = parse_cpulist(f.read()) & os.sched_getaffinity(0)
+        if cpus:
+            os.sched_setaffinity(0, cpus)
+            info.update(bound=True, cpus=len(cpus))
+    except Exception as e:                      # containers may hide the topology: carry on unbound, and say so
+        info["error"] = str(e)
+    return info
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -236,14 +307,57 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32/u8", "data": "synthetic",
-        "config": workload_config(w, args),
+        "config": workload_config(w),
         "cpu_baseline": {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), file=_json_out, flush=True)
 
 
-def workload_config(w, args):
+def run_sharding_dry_run(args):
+    """The multi-rank plumbing of the GPU arm, on CPU: every rank builds its own workload exactly as the GPU arm does
+    (make_workload(args, rank)), resolves a few steps of it with the oracle as the per-rank worker, and the ranks
+    aggregate over gloo the way the GPU arm does over NCCL.  Used by the tests; not a benchmark."""
+    import torch.distributed as dist
+    from oracle import Oracle, FLAG_NO_BYTES
+    from paper_2608_07009_b200 import inputs, sharding
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if "WORLD_SIZE" in os.environ:
+        dist.init_process_group("gloo")
+    w = make_workload(args, rank, steps=args.steps + 1)
+    orc = Oracle(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k, w.entry_bytes, w.capacity,
+                 w.init_len, None, FLAG_NO_BYTES)
+    tr = inputs.Trace(w)
+    n, first_row = 0, None
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        sel, appended, _ = tr.step()
+        if first_row is None:
+            first_row = [int(x) for x in sel[0][0][:4]]
+        if appended:
+            orc.append()
+        for layer in range(w.num_layers):
+            _, h, m = orc.resolve(layer, sel[layer // w.layers_per_group])
+            n += int(h.sum()) + int(m.sum())
+    dt = time.perf_counter() - t0
+    tr.close()
+    orc.close()
+    t_max, n_all = sharding.aggregate(dt, n)
+    rows = [None] * world
+    if "WORLD_SIZE" in os.environ:
+        dist.all_gather_object(rows, first_row)
+        dist.barrier()
+        dist.destroy_process_group()
+    else:
+        rows = [first_row]
+    if rank == 0:
+        print(json.dumps({"impl": "sharding-dry-run", "n_gpus": world, "value": n_all / t_max, "unit": UNIT,
+                          "selections": n_all, "selections_rank0": n, "first_rows": rows,
+                          "config": workload_config(w)}), file=_json_out, flush=True)
+
+
+def workload_config(w):
     return {"workload": w.name, "num_requests": w.num_requests, "num_layers": w.num_layers,
             "layers_per_group": w.layers_per_group, "top_k": w.top_k, "cache_slots": w.cache_slots,
             "entry_bytes": w.entry_bytes, "context": max(w.init_len), "keep": w.keep,
@@ -257,55 +371,6 @@ def workload_config(w, args):
 _json_out = sys.stdout
 
 
-def all_hit_point(dev, hbm_peak):
-    """Scaled all-hit metadata point: 2048 requests x k=2048 x B=4096, rows repeated so that every
-    selection hits; L2 flushed between launches; per-launch CUDA-event time."""
-    import torch
-    import paper_2608_07009_b200 as hs
-    from paper_2608_07009_b200 import inputs
-    w = inputs.scaled_all_hit()
-    N, k, B, E = w.num_requests, w.top_k, w.cache_slots, w.entry_bytes
-    cap = w.capacity
-    hist = [hs.HostHistory(1, cap[r], E) for r in range(N)]
-    for r, h in enumerate(hist):
-        inputs.fill_history(h.ptr, r, 1, cap[r], 0, w.init_len[r], E, w.seed, threads=1)
-    gpu = hs.HiSparse(N, 1, 1, B, k, E, cap, w.init_len, hist, device=dev.index)
-    tr = inputs.Trace(w)
-    sel, _, _ = tr.step()
-    tr.close()
-    sel_d = torch.from_numpy(np.ascontiguousarray(sel[0])).to(dev)
-    tab = torch.empty((N, k), dtype=torch.int32, device=dev)
-    hits = torch.empty(N, dtype=torch.int32, device=dev)
-    misses = torch.empty(N, dtype=torch.int32, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    gpu.resolve(0, sel_d, tab, hits, misses)          # cold: everything misses
-    times = []
-    for i in range(3 + 10):
-        flush.zero_()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        gpu.resolve(0, sel_d, tab, hits, misses)
-        e1.record()
-        e1.synchronize()
-        if i >= 3:
-            times.append(e0.elapsed_time(e1) * 1e-3)
-    assert int(misses.sum().item()) == 0 and int(hits.sum().item()) == N * k
-    geo = gpu.launch_geometry()
-    gpu.close()
-    for h in hist:
-        h.free()
-    t = statistics.mean(times)
-    achieved = ALGO_BYTES_PER_HIT * N * k / t / 1e9
-    return {"bound": "hbm", "achieved": achieved, "peak": hbm_peak["value"], "unit": "GB/s",
-            "frac": achieved / hbm_peak["value"], "peak_source": hbm_peak["source"],
-            "traffic": 76281344 if N == 2048 else None,
-            "traffic_source": "profiles/resolve_kernel_all_hit_set_full.md",
-            "issue_bound_note": "ncu: 47 % of peak instruction issue, 17 % of DRAM throughput: issue/latency bound",
-            "workload": "scaled all-hit point: %d requests x 1 layer, k=%d, B=%d, every selection hits" % (N, k, B),
-            "algorithmic_bytes_per_launch": ALGO_BYTES_PER_HIT * N * k, "launch_us": t * 1e6,
-            "selections_per_s": N * k / t, "ctas_per_request": geo["ctas_per_request"]}
-
-
 def hbm_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -314,30 +379,143 @@ def hbm_peak():
     return {"value": 6650.0, "source": "of fallback (6.65 TB/s)"}
 
 
-def run_ours(args):
+def profile_figure(fname: str, key: str):
+    """A figure that one committed ncu summary states on a line `key: <number> ...` (None when absent), with the
+    commit the summary says it was captured at, so that the number cannot silently outlive the kernel it describes."""
+    path = os.path.join(ROOT, "profiles", fname)
+    try:
+        with open(path) as f:
+            text = f.read()
+    except OSError:
+        return None, None
+    m = re.search(r"^%s:\s*([0-9.eE+]+)" % re.escape(key), text, re.M)
+    c = re.search(r"^captured_at_commit:\s*(\S+)", text, re.M)
+    return (float(m.group(1)) if m else None), (c.group(1) if c else None)
+
+
+class Flusher:
+    """Empties L2 between timed launches.  `clean`: after the 256 MiB write, read another 256 MiB so that the lines
+    left in L2 are clean (otherwise the timed kernel also pays for writing the flusher's dirty lines back)."""
+
+    def __init__(self, dev, clean: bool):
+        import torch
+        self.w = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        self.r = torch.zeros(256 << 18, dtype=torch.int32, device=dev) if clean else None
+
+    def __call__(self):
+        self.w.zero_()
+        if self.r is not None:
+            self.r.sum()
+
+
+def all_hit_points(dev, peak, sm_count):
+    """The all-hit metadata path against HBM bandwidth, on scaled batches (k=2048, B=4096, every selection hits).
+
+    steady: 8192 requests, launches back to back with no flush: one launch reads and writes ~390 MB, three times L2,
+            so nothing a launch touches is still cached when the next one comes to it; launch and ramp-up are
+            amortised as they are in a decode loop.  This is the roofline figure.
+    flushed: 2048 requests, one launch per timing, L2 emptied (256 MiB write, then 256 MiB read) before each: the
+            survey's point; a third of its time is launch, code fetch and ramp-up of a cold kernel.
+    """
+    import torch
+    import paper_2608_07009_b200 as hs
+    from paper_2608_07009_b200 import inputs
+
+    def one(N, timing):
+        w = inputs.scaled_all_hit(N)
+        k, B, E = w.top_k, w.cache_slots, w.entry_bytes
+        cap = w.capacity
+        per = cap[0] * E
+        big = hs.HostHistory(1, N * cap[0], E)              # one pinned buffer, a slice per request (bytes never compared)
+        gpu = hs.HiSparse(N, 1, 1, B, k, E, cap, w.init_len, [big.ptr + r * per for r in range(N)], device=dev.index)
+        tr = inputs.Trace(w)
+        sel, _, _ = tr.step()
+        tr.close()
+        sel_d = torch.from_numpy(np.ascontiguousarray(sel[0])).to(dev)
+        tab = torch.empty((N, k), dtype=torch.int32, device=dev)
+        hits = torch.empty(N, dtype=torch.int32, device=dev)
+        misses = torch.empty(N, dtype=torch.int32, device=dev)
+        gpu.resolve(0, sel_d, tab, hits, misses)          # cold: everything misses
+        times = timing(lambda: gpu.resolve(0, sel_d, tab, hits, misses))
+        torch.cuda.synchronize()
+        assert int(misses.sum().item()) == 0 and int(hits.sum().item()) == N * k
+        geo = gpu.launch_geometry()
+        gpu.close()
+        big.free()
+        return statistics.mean(times), min(times), geo, N * k
+
+    def steady(launch):
+        reps, out = 20, []
+        for _ in range(3):
+            launch()
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                launch()
+            e1.record()
+            e1.synchronize()
+            out.append(e0.elapsed_time(e1) * 1e-3 / reps)
+        return out
+
+    flush = Flusher(dev, clean=True)
+
+    def flushed(launch):
+        out = []
+        for i in range(3 + 10):
+            flush()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            launch()
+            e1.record()
+            e1.synchronize()
+            if i >= 3:
+                out.append(e0.elapsed_time(e1) * 1e-3)
+        return out
+
+    t_s, t_s_min, geo, n_s = one(8192, steady)
+    t_f, t_f_min, _, n_f = one(2048, flushed)
+    ach = ALGO_BYTES_PER_HIT * n_s / t_s / 1e9
+    traffic, commit = profile_figure("resolve_kernel_all_hit.md", "dram_bytes_per_request")
+    res = {"bound": "hbm", "achieved": ach, "peak": peak["value"], "unit": "GB/s", "frac": ach / peak["value"],
+           "peak_source": peak["source"], "kernel": "resolve_kernel (looping narrow blocks)",
+           "workload": "scaled all-hit point: 8192 requests x 1 layer, k=2048, B=4096, every selection hits; 20 launches "
+                       "back to back per timing, no flush: a launch touches ~390 MB (3x L2), so its inputs are not cached",
+           "algorithmic_bytes_per_launch": ALGO_BYTES_PER_HIT * n_s, "launch_us": t_s * 1e6,
+           "selections_per_s": n_s / t_s, "launch_geometry": geo,
+           "traffic": traffic * 8192 if traffic else None,
+           "traffic_source": "profiles/resolve_kernel_all_hit.md: dram__bytes_read + dram__bytes_write per request of a "
+                             "2048-request launch, scaled by the requests of this launch (commit %s)" % commit,
+           "frac_dram_bytes": (traffic * 8192 / t_s / 1e9 / peak["value"]) if traffic else None,
+           "flushed_2048": {"launch_us": t_f * 1e6, "launch_us_min": t_f_min * 1e6,
+                            "achieved": ALGO_BYTES_PER_HIT * n_f / t_f / 1e9,
+                            "frac": ALGO_BYTES_PER_HIT * n_f / t_f / 1e9 / peak["value"],
+                            "workload": "2048 requests, one launch per timing, L2 emptied before each (256 MiB write, then "
+                                        "256 MiB read so that the lines left behind are clean)"}}
+    return res
+
+
+def measure(args, w, dev, local, K, W, full, launched, rank):
+    """Runs workload `w` on this rank's GPU: cold step, W warm-up steps, K timed steps (one CUDA-graph replay each, L2
+    flushed in between), the all-hit replay of the last rows and, with `full`, the per-launch eager pass, the
+    end-to-end pass and the consumer stand-in.  Returns a dict of figures."""
     import torch
     import torch.distributed as dist
     import paper_2608_07009_b200 as hs
     from paper_2608_07009_b200 import inputs, sharding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    launched = "WORLD_SIZE" in os.environ          # under torchrun, also with a single rank
-    if launched:
-        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")   # keep stdout to the one JSON line
-        dist.init_process_group("nccl", device_id=dev)
-
-    w = make_workload(args, rank)
     N, L, lpg, G, k, B, E = (w.num_requests, w.num_layers, w.layers_per_group, w.num_groups, w.top_k,
                              w.cache_slots, w.entry_bytes)
     cap = w.capacity
     t_setup = time.time()
-    hist = [hs.HostHistory(L, cap[r], E) for r in range(N)]
+    hist = []
+    try:
+        for r in range(N):
+            hist.append(hs.HostHistory(L, cap[r], E))
+    except hs.HiSparseError:
+        for h in hist:
+            h.free()
+        raise
     for r, h in enumerate(hist):
         inputs.fill_history(h.ptr, r, L, cap[r], 0, w.init_len[r], E, w.seed)
     flags = (hs.FLAG_SKIP_IO if args.skip_io else 0) | (hs.FLAG_PHASE_TIMERS if args.phases else 0) \
@@ -346,17 +524,11 @@ def run_ours(args):
     gpu = hs.HiSparse(N, L, lpg, B, k, E, cap, w.init_len, hist, device=local, flags=flags,
                       ctas_per_request=args.ctas_per_request)
     geo = gpu.launch_geometry()
-    link_peak = hs.host_link_probe(local, 1 << 30, 10)
-    # ceiling for reads issued by SMs: a copy-only kernel over random records of request 0's history
-    hb = min(hist[0].nbytes, 1 << 32)
-    sm_read = {"%dMB" % mb: hs.scatter_read_probe(hist[0].ptr, hb, E, max(1, (mb << 20) // E), 148, 5, local)
-               for mb in (4, 32)}
 
     # the whole trace, generated up front: cold step, warm-up, timed, eager-profile and e2e steps
-    K, W = args.steps, args.warmup
-    KE = min(K, 8)
+    KE = min(K, 8) if full else 0
     n_dev = 1 + W + K + KE
-    n_steps = n_dev + (1 + K)
+    n_steps = n_dev + ((1 + K) if full else 0)
     tr = inputs.Trace(w)
     sels, kvs = [], []
     for _ in range(n_steps):
@@ -373,7 +545,7 @@ def run_ours(args):
     miss_st = torch.zeros((L, N), dtype=torch.int32, device=dev)
     hits = torch.zeros((n_dev, L, N), dtype=torch.int32, device=dev)
     misses = torch.zeros((n_dev, L, N), dtype=torch.int32, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush = Flusher(dev, clean=False)
     main = torch.cuda.Stream(device=dev)
     side = torch.cuda.Stream(device=dev)
     use_prefetch = lpg > 1 and not args.no_prefetch
@@ -403,7 +575,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if launched:
+        if launched and full:
             dist.barrier()
             torch.cuda.synchronize()
 
@@ -445,7 +617,7 @@ def run_ours(args):
         # NOTE: capturing enqueued nothing; the captured steps run only when replayed.
         for i in range(1, 1 + W):
             load_step(i)
-            flush.zero_()
+            flush()
             graphs[kv_dev[i] is not None].replay()
             save_counts(i)
         barrier()
@@ -456,7 +628,7 @@ def run_ours(args):
         for s_ in range(K):
             i = 1 + W + s_
             load_step(i)
-            flush.zero_()
+            flush()
             step_ev[s_][0].record(main)
             graphs[kv_dev[i] is not None].replay()
             step_ev[s_][1].record(main)
@@ -471,20 +643,30 @@ def run_ours(args):
         for s_ in range(KE):
             i = 1 + W + K + s_
             load_step(i)
-            flush.zero_()
+            flush()
             enqueue_step(kv_dev[i] is not None, lay_ev[s_], stream=main)
             save_counts(i)
         torch.cuda.synchronize()
     step_s = [a.elapsed_time(b_) * 1e-3 for a, b_ in step_ev]
     total_s = sum(step_s)
     anchor_layers = [l for l in range(L) if l % lpg == 0]
-    res_us = np.array([[lay_ev[s_][l][0].elapsed_time(lay_ev[s_][l][1]) * 1e3 for l in range(L)] for s_ in range(KE)])
     hits_h = hits[1 + W:1 + W + K].cpu().numpy().astype(np.int64)
     miss_h = misses[1 + W:1 + W + K].cpu().numpy().astype(np.int64)
     sel_count = int(hits_h.sum() + miss_h.sum())                       # every layer's table entries
     fetched = int(miss_h.sum()) * E                                     # anchors + replays into shared layers
+    out = {"K": K, "W": W, "N": N, "L": L, "lpg": lpg, "E": E, "total_s": total_s, "sel_count": sel_count,
+           "fetched": fetched, "launches": launches, "clocks": clocks, "cold_ms": cold_ms, "geo": geo,
+           "setup_s": setup_s, "pinned_bytes": sum(h.nbytes for h in hist), "use_prefetch": use_prefetch,
+           "misses_per_request_layer": float(miss_h[:, anchor_layers].mean())}
+    if KE:
+        res_us = np.array([[lay_ev[s_][l][0].elapsed_time(lay_ev[s_][l][1]) * 1e3 for l in range(L)] for s_ in range(KE)])
+        out["per_layer"] = {"eager_median": float(np.median(res_us[:, anchor_layers])),
+                            "eager_p99": float(np.percentile(res_us[:, anchor_layers], 99)),
+                            "eager_mean": float(res_us[:, anchor_layers].mean())}
+        if lpg > 1:
+            sh = [l for l in range(L) if l % lpg]
+            out["shared_layer"] = {"median": float(np.median(res_us[:, sh])), "mean": float(res_us[:, sh].mean())}
     status = gpu.status()
-    phases = None
     if args.phases:
         st = gpu.phase_times().astype(np.int64)
         phases = {"pre_fetch_metadata": float((st[:, 3] - st[:, 0]).mean() / 1e3),
@@ -494,50 +676,50 @@ def run_ours(args):
                   "unit": "us, mean over requests, last anchor launch"}
         cyc = st[:, [15, 8, 9, 10, 11, 12, 13, 14]]
         phases["cycles_issue_landed_lookup_dedup_missscan_victims_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
+        out["phases"] = phases
 
-    total_s_max, sel_total = sharding.aggregate(total_s, sel_count, dev)
-
-    # ---- e2e: the following steps through the public API with the inputs in pinned host memory ----
-    sel_pin = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in sels[n_dev:]]
-    kv_pin = [torch.from_numpy(x).pin_memory() if x is not None else None for x in kvs[n_dev:]]
-    cnt_host = torch.empty((2, L, N), dtype=torch.int32).pin_memory()
-    e2e_sel, e2e_s, h2d, d2h = 0, 0.0, 0, 0
-    with torch.cuda.stream(main):
-        for s_ in range(1 + K):
-            flush.zero_()
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            sel_st.copy_(sel_pin[s_], non_blocking=True)
-            nb = sel_pin[s_].numel() * 4
-            if kv_pin[s_] is not None:
-                kv_st.copy_(kv_pin[s_], non_blocking=True)
-                nb += kv_pin[s_].numel()
-            graphs[kv_pin[s_] is not None].replay()
-            cnt_host[0].copy_(hits_st, non_blocking=True)
-            cnt_host[1].copy_(miss_st, non_blocking=True)
-            torch.cuda.synchronize()
-            dt = time.perf_counter() - t0
-            if s_ >= 1:
-                e2e_s += dt
-                e2e_sel += int(cnt_host.sum().item())
-                h2d += nb
-                d2h += cnt_host.numel() * 4
-    h2d //= max(1, K)
-    d2h //= max(1, K)
-    e2e_s, e2e_sel = sharding.aggregate(e2e_s, e2e_sel, dev)
+    if full:
+        out["total_s_max"], out["sel_total"] = sharding.aggregate(total_s, sel_count, dev)
+        # ---- e2e: the following steps through the public API with the inputs in pinned host memory ----
+        sel_pin = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in sels[n_dev:]]
+        kv_pin = [torch.from_numpy(x).pin_memory() if x is not None else None for x in kvs[n_dev:]]
+        cnt_host = torch.empty((2, L, N), dtype=torch.int32).pin_memory()
+        e2e_sel, e2e_s, h2d, d2h = 0, 0.0, 0, 0
+        with torch.cuda.stream(main):
+            for s_ in range(1 + K):
+                flush()
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                sel_st.copy_(sel_pin[s_], non_blocking=True)
+                nb = sel_pin[s_].numel() * 4
+                if kv_pin[s_] is not None:
+                    kv_st.copy_(kv_pin[s_], non_blocking=True)
+                    nb += kv_pin[s_].numel()
+                graphs[kv_pin[s_] is not None].replay()
+                cnt_host[0].copy_(hits_st, non_blocking=True)
+                cnt_host[1].copy_(miss_st, non_blocking=True)
+                torch.cuda.synchronize()
+                dt = time.perf_counter() - t0
+                if s_ >= 1:
+                    e2e_s += dt
+                    e2e_sel += int(cnt_host.sum().item())
+                    h2d += nb
+                    d2h += cnt_host.numel() * 4
+        out["h2d"], out["d2h"] = h2d // max(1, K), d2h // max(1, K)
+        out["e2e_s"], out["e2e_sel"] = sharding.aggregate(e2e_s, e2e_sel, dev)
     # ---- the same rows once more, without an append: every selection hits (the residual cost of a layer-resolve
     # when nothing has to be fetched, at the workload's own size) ----
-    hit_only = None
+    out["hit_only"] = None
     if not args.skip_io:
         with torch.cuda.stream(main):
             torch.cuda.synchronize()
             gph = torch.cuda.CUDAGraph()
             gph.capture_begin()
-            n_hit_launch = enqueue_step(False, stream=main)
+            enqueue_step(False, stream=main)
             gph.capture_end()
             ts = []
             for i in range(3 + 10):
-                flush.zero_()
+                flush()
                 a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(main)
                 gph.replay()
@@ -549,19 +731,19 @@ def run_ours(args):
             n_sel_hit = int(hits_st.sum().item())
             if int(miss_st.sum().item()) == 0:
                 t_hit = statistics.mean(ts)
-                hit_only = {"launch_us": t_hit / L * 1e6, "selections_per_s": n_sel_hit / t_hit,
-                            "hbm_gb_s_algorithmic": ALGO_BYTES_PER_HIT * n_sel_hit / t_hit / 1e9,
-                            "note": "graph of %d resolves on the last step's rows, no append, L2 flushed between replays"
-                                    % L}
+                out["hit_only"] = {"launch_us": t_hit / L * 1e6, "selections_per_s": n_sel_hit / t_hit,
+                                   "hbm_gb_s_algorithmic": ALGO_BYTES_PER_HIT * n_sel_hit / t_hit / 1e9,
+                                   "note": "graph of %d resolves on the last step's rows, no append, L2 flushed between "
+                                           "replays" % L}
             del gph
     # ---- the consumer's gather (stand-in for sparse attention reading the cache through the slot table) ----
-    consumer = None
-    if not args.skip_io and N * k * E <= (2 << 30):
+    out["consumer"] = None
+    if full and not args.skip_io and N * k * E <= (2 << 30):
         with torch.cuda.stream(main):
             out_buf = torch.empty((N, k, E), dtype=torch.uint8, device=dev)
             ts = []
             for i in range(3 + 8):
-                flush.zero_()
+                flush()
                 a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(main)
                 gpu.gather(0, tabs[0], out_buf, stream=main)
@@ -571,20 +753,101 @@ def run_ours(args):
                     ts.append(a.elapsed_time(b_) * 1e-3)
             t_g = statistics.mean(ts)
             peak = hbm_peak()
-            consumer = {"kernel": "gather_kernel", "launch_us": t_g * 1e6, "bytes_read_plus_written": 2 * N * k * E,
-                        "hbm_gb_s": 2 * N * k * E / t_g / 1e9, "frac_of_hbm_peak": 2 * N * k * E / t_g / 1e9 / peak["value"],
-                        "peak_source": peak["source"]}
+            out["consumer"] = {"kernel": "gather_kernel", "launch_us": t_g * 1e6, "bytes_read_plus_written": 2 * N * k * E,
+                               "hbm_gb_s": 2 * N * k * E / t_g / 1e9,
+                               "frac_of_hbm_peak": 2 * N * k * E / t_g / 1e9 / peak["value"], "peak_source": peak["source"]}
             del out_buf
-    status |= gpu.status()
+    out["status"] = status | gpu.status()
+    out["sm_read"] = None
+    if full:
+        # ceiling for reads issued by SMs: a copy-only kernel over random records of request 0's history
+        hb = min(hist[0].nbytes, 1 << 32)
+        sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+        out["sm_read"] = {"%dMB" % mb: hs.scatter_read_probe(hist[0].ptr, hb, E, max(1, (mb << 20) // E), sm_count, 5, local)
+                          for mb in (4, 32)}
     del graphs
     gpu.close()
     for h in hist:
         h.free()
+    return out
+
+
+def per_config_runs(args, dev, local, link_peak):
+    """Short runs of the other miss-heavy configurations (a few steps each), so that every configuration's
+    per-launch figure and its all-hit replay are on the same line as the default workload's."""
+    import copy
+    import paper_2608_07009_b200 as hs
+    res = {}
+    K, W = 6, 2
+    plan = [("c3", "c3_dsa_long, 50 % overlap, exact prefetch", dict(overlap=0.5)), ("c4", "c4_nsa_blocks", {}),
+            ("c5", "c5_quest_pages", {})]
+    for name, label, over in plan:
+        a = copy.copy(args)
+        a.requests = a.layers = a.cache_slots = a.top_k = 0
+        a.phases = a.skip_io = a.spec_hint = False
+        for kk, vv in over.items():
+            setattr(a, kk, vv)
+        entry = {"workload": label}
+        for layers in (0, 4):                       # the configuration's own layer count first, 4 layers if that cannot be pinned
+            a.layers = layers
+            w = make_workload(a, 0, name, steps=1 + W + K + 1)
+            try:
+                m = measure(a, w, dev, local, K, W, False, False, 0)
+            except hs.HiSparseError as e:
+                if e.code != hs.ENOMEM or layers:
+                    entry["error"] = str(e)
+                    break
+                entry["reduced"] = "the host could not pin %d layers of history (%.1f GB): 4 layers instead, every other " \
+                                   "dimension as configured" % (w.num_layers, w.host_bytes() / 1e9)
+                continue
+            n_launch = m["K"] * m["L"]
+            launch_s = m["total_s"] / n_launch
+            ach = m["fetched"] / n_launch / launch_s / 1e9
+            entry.update({"num_requests": m["N"], "num_layers": m["L"], "layers_per_group": m["lpg"], "steps": K,
+                          "warmup": W, "launch_us": launch_s * 1e6, "fetched_bytes_per_launch": m["fetched"] / n_launch,
+                          "h2d_gb_s": ach, "frac": ach / link_peak if link_peak else None,
+                          "selections_per_s": m["sel_count"] / m["total_s"],
+                          "misses_per_request_layer": m["misses_per_request_layer"], "status_bits": m["status"],
+                          "hit_only_step": m["hit_only"], "launch_geometry": m["geo"], "pinned_bytes": m["pinned_bytes"],
+                          "setup_s": m["setup_s"], "prefetch": m["use_prefetch"], "cold_step_ms": m["cold_ms"]})
+            break
+        res[name] = entry
+    return res
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2608_07009_b200 as hs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    placement = bind_near_gpu(local)               # before any pinned allocation
+    launched = "WORLD_SIZE" in os.environ          # under torchrun, also with a single rank
+    if launched:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")                # communicator / rank lines, for the record
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")   # keep stdout to the one JSON line
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = make_workload(args, rank)
+    K, W = args.steps, args.warmup
+    link_peak = hs.host_link_probe(local, 1 << 30, 10)
+    m = measure(args, w, dev, local, K, W, True, launched, rank)
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
 
     extra = {}
+    if rank == 0 and world == 1 and not args.no_per_config and args.workload == "c2" and not (
+            args.requests or args.layers or args.cache_slots or args.top_k or args.context or args.skip_io):
+        extra["per_config"] = per_config_runs(args, dev, local, link_peak)
     if rank == 0 and not args.no_all_hit:
-        extra["roofline_all_hit"] = all_hit_point(dev, hbm_peak())
+        extra["roofline_all_hit"] = all_hit_points(dev, hbm_peak(), sm_count)
     if rank == 0 and not args.no_cpu_baseline:
+        N, L = w.num_requests, w.num_layers
         n_req = min(args.cpu_sample_requests, N)
         steps_cpu = args.cpu_sample_steps
         rate, _, _ = oracle_throughput(w, n_req, steps_cpu, 1)
@@ -592,7 +855,7 @@ def run_ours(args):
             "value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": "requests 0..%d of %d, all %d layers, %d steps after the cold step and 1 warm-up step" % (
                 n_req - 1, N, L, steps_cpu)}
-        threads = min(os.cpu_count() or 1, N)
+        threads = min(len(os.sched_getaffinity(0)) or 1, N)
         n_par = min(N, threads)
         extra["cpu_baseline_parallel"] = {
             "value": oracle_throughput_parallel(w, n_par, max(1, steps_cpu // 4), threads), "unit": UNIT,
@@ -608,17 +871,21 @@ def run_ours(args):
     # the dominant kernel is the Resolve launch of an anchor layer; its average duration is the CUDA-event time
     # of a step's graph replay divided by the number of resolve launches in it (the append's two small kernels
     # are charged to it, so the figure is on the safe side)
-    n_launch = K * L
-    avg_launch_s = total_s / n_launch
-    algo_bytes_per_launch = fetched / n_launch
+    n_launch = K * m["L"]
+    avg_launch_s = m["total_s"] / n_launch
+    algo_bytes_per_launch = m["fetched"] / n_launch
     achieved = algo_bytes_per_launch / avg_launch_s / 1e9 if avg_launch_s > 0 else 0.0
+    is_c2 = (w.name, m["N"]) == ("c2_dsa_decode", 32)
+    dram, commit = profile_figure("resolve_kernel_c2.md", "dram_bytes_per_launch")
+    pcie, _ = profile_figure("resolve_kernel_c2.md", "pcie_read_bytes_per_launch")
     line = {
-        "metric": METRIC, "value": sel_total / total_s_max, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": total_s_max / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32/u8", "data": "synthetic", "config": workload_config(w, args),
-        "e2e": {"value": e2e_sel / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches,
-        "clocks": clocks,
+        "metric": METRIC, "value": m["sel_total"] / m["total_s_max"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": m["total_s_max"] / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32/u8", "data": "synthetic", "config": workload_config(w),
+        "e2e": {"value": m["e2e_sel"] / m["e2e_s"], "unit": UNIT, "h2d_bytes_per_step": m["h2d"],
+                "d2h_bytes_per_step": m["d2h"]},
+        "gpu_launches": m["launches"],
+        "clocks": m["clocks"],
         "roofline": {
             "bound": "host_link", "bound_note": "the fetch over the host link (PCIe Gen5 x16) bounds a miss-heavy resolve, "
             "neither HBM nor the tensor cores; the all-hit path is reported against HBM in roofline_all_hit",
@@ -626,31 +893,38 @@ def run_ours(args):
             "frac": achieved / link_peak if link_peak else None,
             "peak_source": "measured in this run: best of 10 bulk pinned cudaMemcpyAsync H2D of 1 GiB",
             "kernel": "resolve_kernel",
-            "traffic": 2883328 if (w.name, N) == ("c2_dsa_decode", 32) else None,
-            "traffic_source": "profiles/resolve_kernel_c2_set_full.md: dram__bytes_read + dram__bytes_write of one launch",
+            "traffic": dram if is_c2 else None,
+            "traffic_host_link": pcie if is_c2 else None,
+            "traffic_source": "profiles/resolve_kernel_c2.md (commit %s): dram__bytes_read + dram__bytes_write, and "
+                              "pcie__read_bytes, of one launch of this shape; the fetched records cross the host link and "
+                              "stay in L2, so the host-link figure is the meaningful one" % commit,
             "algorithmic_bytes_per_launch": algo_bytes_per_launch, "launch_us": avg_launch_s * 1e6,
             "launch_us_method": "CUDA events around each step's graph replay / resolve launches per step"},
-        "per_layer_resolve_us": {"graph": avg_launch_s * 1e6,
-                                 "eager_median": float(np.median(res_us[:, anchor_layers])),
-                                 "eager_p99": float(np.percentile(res_us[:, anchor_layers], 99)),
-                                 "eager_mean": float(res_us[:, anchor_layers].mean())},
-        "misses_per_request_layer": float(miss_h[:, anchor_layers].mean()),
-        "host_link": {"memcpy_peak_gb_s": link_peak, "sm_issued_read_gb_s": sm_read,
-                      "note": "copy-only kernel, 148 blocks, random records of this workload's size"},
-        "cold_step_ms": cold_ms, "hit_only_step": hit_only, "consumer_gather": consumer, "status_bits": status, "launch_geometry": geo, "setup_s": setup_s,
+        "per_layer_resolve_us": dict(graph=avg_launch_s * 1e6, **m.get("per_layer", {})),
+        "misses_per_request_layer": m["misses_per_request_layer"],
+        "host_link": {"memcpy_peak_gb_s": link_peak, "sm_issued_read_gb_s": m["sm_read"],
+                      "note": "copy-only kernel, one block per SM, random records of this workload's size"},
+        "placement": placement,
+        "cold_step_ms": m["cold_ms"], "hit_only_step": m["hit_only"], "consumer_gather": m["consumer"],
+        "status_bits": m["status"], "launch_geometry": m["geo"], "setup_s": m["setup_s"], "pinned_bytes": m["pinned_bytes"],
     }
-    if phases:
-        line["phases_us"] = phases
-    if lpg > 1:
-        sh = [l for l in range(L) if l % lpg]
-        line["shared_layer_resolve_us"] = {"median": float(np.median(res_us[:, sh])), "mean": float(res_us[:, sh].mean())}
-        line["prefetch"] = use_prefetch
+    if "phases" in m:
+        line["phases_us"] = m["phases"]
+    if "shared_layer" in m:
+        line["shared_layer_resolve_us"] = m["shared_layer"]
+        line["prefetch"] = m["use_prefetch"]
     line.update(extra)
     print(json.dumps(line), file=_json_out, flush=True)
 
 
-def main():
-    args = parse_args()
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
+    args = parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_ranks(args, argv))
+    if args.gpus > 1 and "WORLD_SIZE" in os.environ and int(os.environ["WORLD_SIZE"]) != args.gpus and args.impl == "ours":
+        print("bench.py: --gpus %d but the launcher started %s ranks" % (args.gpus, os.environ["WORLD_SIZE"]), file=sys.stderr)
+        sys.exit(2)
     # stdout carries exactly one JSON line: whatever a library writes to file descriptor 1 (NCCL's version banner
     # under torchrun, for one) goes to stderr instead
     global _json_out
@@ -659,6 +933,8 @@ def main():
     os.dup2(2, 1)
     if args.impl == "reference":
         run_reference(args)
+    elif args.impl == "sharding-dry-run":
+        run_sharding_dry_run(args)
     else:
         run_ours(args)
 

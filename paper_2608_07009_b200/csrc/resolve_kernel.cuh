@@ -28,6 +28,28 @@ __device__ __forceinline__ int block_scan_excl(int v, int *s_warp, int &total) {
   return warp_excl + incl - v;
 }
 
+// Block-wide exclusive rank over NB flag bits per thread, thread-major (thread t's bits 0..NB-1 come before thread
+// t+1's): returns the number of set bits in all earlier threads.  Ballots and population counts instead of shuffle
+// scans; one barrier.  s_warp: 32 ints of scratch, not to be reused before the block has passed another barrier.
+template <int NB>
+__device__ __forceinline__ int block_rank_bits(const uint32_t bits, int *s_warp, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const uint32_t lt = (1u << lane) - 1u;
+  int below = 0, wtot = 0;
+#pragma unroll
+  for (int i = 0; i < NB; ++i) {
+    const uint32_t b = __ballot_sync(0xffffffffu, (bits >> i) & 1u);
+    below += __popc(b & lt);
+    wtot += __popc(b);
+  }
+  if (lane == 0) s_warp[warp] = wtot;
+  __syncthreads();
+  const int w = lane < nw ? s_warp[lane] : 0;
+  const int before = __reduce_add_sync(0xffffffffu, lane < warp ? w : 0);
+  total = __reduce_add_sync(0xffffffffu, w);
+  return before + below;
+}
+
 // Asynchronous global -> shared staging (cp.async, 16 bytes per thread and step); falls back to plain 4- or
 // 2-byte copies when the size or an address is not a multiple of 16.  Complete after cp.async.wait_all + barrier.
 __device__ __forceinline__ void stage_async(void *smem_dst, const void *gmem_src, int bytes) {
@@ -408,6 +430,11 @@ __device__ __forceinline__ void stage_issue(const DevState &d, const SmemView &v
   }
 }
 
+// How a repeated missing position is caught (list_misses): through claims in the staged page-table slice, which
+// lookup_phase has already stored (kClaimsStored) or list_misses still has to store (kClaimsPending), or, when the
+// slice is not in shared memory, through the table of missing positions (kClaimsNone).
+constexpr int kClaimsNone = 0, kClaimsStored = 1, kClaimsPending = 2;
+
 // Phase 2 of Sec. 3.4 as the first block of a cluster runs it, up to the block-wide vote "did anything miss?".
 // Thread t owns the KPT consecutive row entries [t*KPT, t*KPT + KPT): it reads them with one vector load, looks them
 // up in the page table, marks the slots that hit, and writes its part of the slot table at once (a hit's slot is final;
@@ -418,7 +445,7 @@ template <int T, int KPT>
 __device__ __forceinline__ void lookup_phase(const DevState &d, const SmemView &v, const SliceGeom &q, const ReqCtx &c,
                                              const uint32_t stage_parity, unsigned long long *stamps,
                                              int32_t (&pos)[KPT], int32_t (&cls)[KPT], uint32_t &my_status, bool &any_miss,
-                                             uint32_t &t_now, uint32_t &order_t) {
+                                             uint32_t &t_now, uint32_t &order_t, int &claims) {
   const int tid = threadIdx.x;
   const int k = d.k, B = d.B;
   const int r = c.r, S = c.S;
@@ -453,11 +480,12 @@ __device__ __forceinline__ void lookup_phase(const DevState &d, const SmemView &
   const bool use_staged = q.staged && !timed_out;
   if (timed_out) my_status |= HISPARSE_STATUS_TIMEOUT;
   if (timers && tid == 0) stamps[9] = clock64();
-  const int16_t *s_p2s = reinterpret_cast<const int16_t *>(v.ring) + q.lead;
+  int16_t *s_p2s = reinterpret_cast<int16_t *>(v.ring) + q.lead;
   if (coop) cluster_lookups<T>(row, q.p2s, k, len, 0, S, v.got);
 
   // Phase 2: hit detection through the page table (position -> slot); all of a thread's lookups are issued
-  // before the first is used.
+  // before the first is used, unconditionally (an entry that is padding or out of range looks up position 0 and
+  // discards the answer).
   const int j0 = tid * KPT;
 #pragma unroll
   for (int i = 0; i < KPT; ++i) pos[i] = -1;
@@ -471,37 +499,45 @@ __device__ __forceinline__ void lookup_phase(const DevState &d, const SmemView &
     }
   }
   int32_t got[KPT];
+  const uint32_t ulen = (uint32_t)len;
+  int bad = 0;
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
     if (j0 + i >= k) pos[i] = -1;
-    const bool ok = pos[i] >= 0 && (int64_t)pos[i] < len;
-    if (pos[i] != -1 && !ok) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
-    if (!ok) pos[i] = -1;
-    got[i] = !ok ? -1 : (int32_t)(use_staged ? s_p2s[pos[i]] : coop ? v.got[j0 + i] : __ldg(q.p2s + pos[i]));
+    const bool ok = (uint32_t)pos[i] < ulen;  // 0 <= p < len (positions and lengths fit 31 bits)
+    bad |= (!ok) & (pos[i] != -1);
+    const int32_t idx = ok ? pos[i] : 0;
+    const int32_t raw = use_staged ? (int32_t)s_p2s[idx] : coop ? (int32_t)v.got[j0 + i < k ? j0 + i : 0] : (int32_t)__ldg(q.p2s + idx);
+    pos[i] = ok ? pos[i] : -1;
+    got[i] = ok ? raw : -1;
   }
+  if (bad) my_status |= HISPARSE_STATUS_OUT_OF_RANGE;
   int miss = 0, nhit = 0;
   int32_t val[KPT];
   const int32_t base = r * (B + 1);
   const uint8_t tag = (uint8_t)c.tag;
+  const int32_t inewest = newest >= 0 ? (int32_t)newest : -2;  // -2: no newest record (a discarded entry is -1)
 #pragma unroll
   for (int i = 0; i < KPT; ++i) {
     const int32_t p = pos[i];
     int32_t o = -1;
-    if (p >= 0) {
-      if ((int64_t)p == newest) {  // reserved newest-record slot, outside the LRU set
-        o = B;
-        if (atomicExch(&s_misc[2], 1) != 0) my_status |= HISPARSE_STATUS_DUPLICATE;
-      } else if (got[i] >= 0) {
-        // A plain byte store marks the slot (shared-memory atomics on a bitset were measured to take about half of
-        // a resolve in which nothing misses).  The hit's stamp is written later, in slot order (coalesced), from
-        // the marks; a resident position selected twice marks one slot twice, which the counts reveal.
-        o = got[i];
-        v.marks[o] = tag;
-        ++nhit;
-      } else {
-        o = kMiss;
-        miss = 1;
-      }
+    if (p == inewest) {  // reserved newest-record slot, outside the LRU set
+      o = B;
+      if (atomicExch(&s_misc[2], 1) != 0) my_status |= HISPARSE_STATUS_DUPLICATE;
+    } else if (got[i] >= 0) {
+      // A plain byte store marks the slot (shared-memory atomics on a bitset were measured to take about half of
+      // a resolve in which nothing misses).  The hit's stamp is written later, in slot order (coalesced), from
+      // the marks; a resident position selected twice marks one slot twice, which the counts reveal.
+      o = got[i];
+      v.marks[o] = tag;
+      ++nhit;
+    } else if (p >= 0) {
+      o = kMiss;
+      miss = 1;
+      // With the slice in shared memory, a missing position is claimed there by its row index: reading the claim
+      // back after the vote tells whether another row entry selected the same position (any negative entry reads
+      // as "not resident", so a claim does not disturb a later lookup of that position).
+      if (use_staged) s_p2s[p] = (int16_t)(-2 - (j0 + i));
     }
     cls[i] = o;
     val[i] = o < 0 ? -1 : base + o;
@@ -528,67 +564,87 @@ __device__ __forceinline__ void lookup_phase(const DevState &d, const SmemView &
   nhit = __reduce_add_sync(0xffffffffu, nhit);
   if ((tid & 31) == 0 && nhit) atomicAdd(&s_misc[1], nhit);
   any_miss = __syncthreads_or(miss) != 0;
+  claims = use_staged ? kClaimsStored : kClaimsNone;
   if (timers && tid == 0) stamps[10] = clock64();
 }
 
-// The rest of what precedes the fetch when something missed: the missing positions go through a table (position ->
-// row index) whose only job is to catch a position that was selected twice, so that it claims one victim, not two;
-// then ONE block scan puts the misses in selection order.  On return plan_pos[i] / missj[i] hold the position and
-// the row index of the i-th miss and m their number.
+// The rest of what precedes the fetch when something missed: catch a missing position that was selected twice (it
+// must claim one victim, not two), then ONE block-wide rank puts the misses in selection order.  On return
+// plan_pos[i] / missj[i] hold the position and the row index of the i-th miss and m their number.
+// Repeated positions are a violation of the caller's contract, so the common case is made cheap: every miss has
+// claimed its position in the staged slice with its row index (a plain store); a claim that reads back as someone
+// else's reveals a repetition, and only then (or when the slice is not in shared memory) do the missing positions go
+// through the table (position -> lowest row index), which decides the owner the way the specification does.
 template <int T, int KPT>
 __device__ __forceinline__ void list_misses(const DevState &d, const SmemView &v, int32_t *trow, int32_t *arow,
-                                            unsigned long long *stamps, int *s_misc,
+                                            unsigned long long *stamps, int *s_misc, int16_t *s_p2s, const int claims,
                                             const int32_t (&pos)[KPT], int32_t (&cls)[KPT], uint32_t &my_status, int &m) {
   const int tid = threadIdx.x;
   const int H = d.H;
   const uint32_t mask = (uint32_t)(H - 1);
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
   const int j0 = tid * KPT;
-  if (d.sm_tab < 0) {  // the table shares the ring's memory and is cleared only now that it is needed
-    for (int i = tid; i < H; i += T) v.tab[i] = kEmptyEntry;
-    __syncthreads();
-  }
+  bool need_table = true;
+  if (claims != kClaimsNone) {
+    if (claims == kClaimsPending) {
 #pragma unroll
-  for (int i = 0; i < KPT; ++i)
-    if (cls[i] == kMiss) {
-      const int32_t p = pos[i];
-      const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)(j0 + i);
-      uint32_t h = hash_pos(p, d.hshift);
-      for (uint32_t it = 0; it <= mask; ++it) {
-        const unsigned long long old = atomicCAS(&v.tab[h], kEmptyEntry, entry);
-        if (old == kEmptyEntry) break;
-        if ((int32_t)(old >> 32) == p) {  // selected twice: the lowest row index owns the entry
-          atomicMin(&v.tab[h], entry);
-          s_misc[0] = 1;
-          break;
-        }
-        h = (h + 1u) & mask;
-      }
+      for (int i = 0; i < KPT; ++i)
+        if (cls[i] == kMiss) s_p2s[pos[i]] = (int16_t)(-2 - (j0 + i));
+      __syncthreads();
     }
-  __syncthreads();
-  if (timers && tid == 0) stamps[11] = clock64();
-  if (s_misc[0]) {  // rare: every later occurrence of a repeated missing position follows the first one
+    int other = 0;
+#pragma unroll
+    for (int i = 0; i < KPT; ++i)
+      if (cls[i] == kMiss) other |= s_p2s[pos[i]] != (int16_t)(-2 - (j0 + i));
+    need_table = __syncthreads_or(other) != 0;  // (also: every claim has been read before the ring is used again)
+  }
+  if (need_table) {
+    if (d.sm_tab < 0) {  // the table shares the ring's memory and is cleared only now that it is needed
+      for (int i = tid; i < H; i += T) v.tab[i] = kEmptyEntry;
+      __syncthreads();
+    }
 #pragma unroll
     for (int i = 0; i < KPT; ++i)
       if (cls[i] == kMiss) {
-        const int32_t key[1] = {pos[i]};
-        int32_t owner[1];
-        table_lookup<1>(v.tab, mask, d.hshift, key, owner);
-        if (owner[0] != j0 + i) {
-          cls[i] = -1;  // not a miss of its own; its table entry is copied from the owner's at the end
-          trow[j0 + i] = kDupBase - owner[0];
-          if (arow) arow[j0 + i] = kDupBase - owner[0];
-          my_status |= HISPARSE_STATUS_DUPLICATE;
+        const int32_t p = pos[i];
+        const unsigned long long entry = ((unsigned long long)(uint32_t)p << 32) | (uint32_t)(j0 + i);
+        uint32_t h = hash_pos(p, d.hshift);
+        for (uint32_t it = 0; it <= mask; ++it) {
+          const unsigned long long old = atomicCAS(&v.tab[h], kEmptyEntry, entry);
+          if (old == kEmptyEntry) break;
+          if ((int32_t)(old >> 32) == p) {  // selected twice: the lowest row index owns the entry
+            atomicMin(&v.tab[h], entry);
+            s_misc[0] = 1;
+            break;
+          }
+          h = (h + 1u) & mask;
         }
       }
+    __syncthreads();
+    if (s_misc[0]) {  // every later occurrence of a repeated missing position follows the first one
+#pragma unroll
+      for (int i = 0; i < KPT; ++i)
+        if (cls[i] == kMiss) {
+          const int32_t key[1] = {pos[i]};
+          int32_t owner[1];
+          table_lookup<1>(v.tab, mask, d.hshift, key, owner);
+          if (owner[0] != j0 + i) {
+            cls[i] = -1;  // not a miss of its own; its table entry is copied from the owner's at the end
+            trow[j0 + i] = kDupBase - owner[0];
+            if (arow) arow[j0 + i] = kDupBase - owner[0];
+            my_status |= HISPARSE_STATUS_DUPLICATE;
+          }
+        }
+    }
   }
+  if (timers && tid == 0) stamps[11] = clock64();
   // Phase 3, first half: the misses in selection order.  Their positions are all the fetch needs to start loading;
   // the victims are only needed when a record is stored.
   uint32_t miss_mask = 0;
 #pragma unroll
   for (int i = 0; i < KPT; ++i)
     if (cls[i] == kMiss) miss_mask |= 1u << i;
-  int mrank = block_scan_excl(__popc(miss_mask), v.warp, m);
+  int mrank = block_rank_bits<KPT>(miss_mask, v.warp, m);
 #pragma unroll
   for (int i = 0; i < KPT; ++i)
     if ((miss_mask >> i) & 1u) {
@@ -596,7 +652,7 @@ __device__ __forceinline__ void list_misses(const DevState &d, const SmemView &v
       v.missj[mrank] = (uint16_t)(j0 + i);
       ++mrank;
     }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the table's memory may be the ring
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the ring was written by this block's threads
   if (timers && tid == 0) stamps[12] = clock64();
   __syncthreads();
 }
@@ -724,7 +780,7 @@ __device__ __forceinline__ void choose_victims(const DevState &d, const SmemView
 // current by every resolve): list the misses, start the fetch, choose the victims while the first loads fly, write the
 // metadata back, rewrite the recency list, then drain the fetch.  pos / cls come from lookup_phase.
 template <int T, int KPT>
-__device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, const int32_t (&pos)[KPT],
+__device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, const int claims, const int32_t (&pos)[KPT],
                                           int32_t (&cls)[KPT], const uint32_t t, const uint32_t order_t,
                                           uint32_t my_status, uint32_t &fetch_parity, uint32_t &order_parity,
                                           bool &gave_up) {
@@ -759,7 +815,8 @@ __device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, co
   } else {
     stage_async(v.order, order_g, B * 2);
   }
-  list_misses<T, KPT>(d, v, c.trow, c.arow, stamps, s_misc, pos, cls, my_status, m);
+  int16_t *s_p2s = reinterpret_cast<int16_t *>(v.ring) + slice_geom(d, c.g, c.cap_r, c.p2s_off_r).lead;
+  list_misses<T, KPT>(d, v, c.trow, c.arow, stamps, s_misc, s_p2s, claims, pos, cls, my_status, m);
   if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
   // Phase 4 starts here, with the positions of the misses: the first batch of host loads is in flight while the
   // victims are chosen (a record's slot is only needed when it is stored) and the metadata is written back
@@ -915,7 +972,8 @@ __device__ __noinline__ void miss_path_cold(const DevState &d, const ReqCtx &c, 
 #pragma unroll
   for (int i = 0; i < KPT; ++i) cls[i] = pos[i] >= 0 ? kMiss : -1;  // only the misses matter from here on
   // (the array gets its real content only after several block barriers: every thread has its entries by then)
-  miss_path<T, KPT>(d, c, pos, cls, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+  const int claims = slice_geom(d, c.g, c.cap_r, c.p2s_off_r).staged ? kClaimsPending : kClaimsNone;
+  miss_path<T, KPT>(d, c, claims, pos, cls, t, order_t, my_status, fetch_parity, order_parity, gave_up);
 }
 
 // A block of a cluster other than the first: shares the page-table lookups when the slice cannot be staged, then
@@ -1057,14 +1115,15 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
   uint32_t state = 0;   // kCold* bits: phases of the fetch / list barriers as the out-of-line path left them
   int tag = 0;
   uint32_t parity = 0;
+  // a request's resolve count is loaded one request ahead (with the next request's inputs), so that the trip to
+  // memory is over when the count is needed
+  uint32_t t_ahead = r < N ? d.t[r * G + g] : 0u;
   // nothing appends while a resolve runs (stream order): the lengths are the same for every request of the launch
   const int na = *(volatile int32_t *)d.n_appends;
   int len = il + na, newest = na > 0 ? il + na - 1 : -2;  // -2: no newest record (a discarded entry is -1)
   if (len > cap) { len = cap; newest = -2; }
-  // a request's resolve count is loaded one request ahead (with the next request's inputs), so that the trip to
-  // memory is over when the count is needed
-  uint32_t t_ahead = r < N ? d.t[r * G + g] : 0u;
-  for (; r < N; r += stride, parity ^= 1u) {
+  bool more = r < N;
+  for (; more; parity ^= 1u) {
     const int rg = r * G + g;                       // N * G fits 32 bits (the metadata arrays are indexed by it)
     const uint32_t a_set = a_misc + parity * 32u;
     if (tag == 255) {
@@ -1105,8 +1164,7 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
     int32_t val[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      // (the newest position is never resident in an LRU slot: its record sits in the reserved slot)
-      const bool isnew = pos[i] == newest, hit = got[i] >= 0;
+      const bool isnew = pos[i] == newest, hit = got[i] >= 0 && !isnew;
       miss |= pos[i] >= 0 && !isnew && !hit;
       sts_u8(hit ? a_marks + (uint32_t)got[i] : a_spare, (uint32_t)tag);
       nhit += hit;
@@ -1125,25 +1183,28 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
     }
     nhit = __reduce_add_sync(0xffffffffu, nhit);
     if (lane == 0 && nhit) red_add_s32(a_set + 4u, nhit);
-    const bool has_next = r + stride < N;
-    if (has_next) t_ahead = d.t[rg + stride * G];
-    if (__syncthreads_or(miss)) {
+    const bool any_miss = __syncthreads_or(miss) != 0;
+    const int rn = r + stride;        // the request this block takes next
+    const bool has_next = rn < N;
+    if (has_next) t_ahead = d.t[rn * G + g];
+    if (any_miss) {
       // something missed: the general path, out of line; the thread's missing positions travel through shared memory
       if (mine) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) sts_s32(a_stash + 4u * i, (pos[i] >= 0 && pos[i] != newest && got[i] < 0) ? pos[i] : -1);
       }
       state = lean_miss<T>(d, layer, g, sel, table, hits_out, misses_out, r, (int)parity, tag, has_next, t, st, state);
-      if (has_next) {  // after a fetch, the next request's inputs can only start once every thread is done with the ring
-        if (__syncthreads_or((state & kColdGaveUp) != 0)) return;
-        if (tid < 32) lean_stage_issue<T>(d, sel, g, r + stride, a_base, a_ring, stage_bar);
-      }
+      // after a fetch, the next request's inputs can only start once every thread is done with the ring
+      if (__syncthreads_or((state & kColdGaveUp) != 0)) break;
+      if (has_next && tid < 32) lean_stage_issue<T>(d, sel, g, rn, a_base, a_ring, stage_bar);
+      more = has_next;
+      r = rn;
       continue;
     }
     if (has_next && !gave_up) {
       // the row and the ring are free (every thread consumed its entries before the vote): the next request's inputs
       // travel while this one's stamps are written
-      if (tid < 32) lean_stage_issue<T>(d, sel, g, r + stride, a_base, a_ring, stage_bar);
+      if (tid < 32) lean_stage_issue<T>(d, sel, g, rn, a_base, a_ring, stage_bar);
     } else {
       asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
@@ -1181,7 +1242,9 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
       if (!stamp_hits) d.order_t[rg] = t;
     }
     if (st) atomicOr(d.status, st);
-    if (gave_up) return;
+    if (gave_up) break;
+    more = has_next;
+    r = rn;
   }
 }
 
@@ -1195,10 +1258,10 @@ __global__ void __launch_bounds__(T, MINB)
 resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_t *__restrict__ sel,
                int32_t *__restrict__ table, int32_t *__restrict__ hits_out, int32_t *__restrict__ misses_out, const int S) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int part = blockIdx.x % S, stride = gridDim.x / S;
   const int g = layer / d.lpg;
-  const int k = d.k, B = d.B, W = d.W;
+  const int k = d.k, B = d.B;
   const bool timers = d.flags & HISPARSE_FLAG_PHASE_TIMERS;
 
   // Prologue that depends on nothing an earlier kernel wrote: barriers, cleared marks (and table, when it has memory
@@ -1274,18 +1337,19 @@ resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_
     }
     uint32_t my_status = 0, order_t = 0, t = 0;
     bool any_miss = false;
+    int claims = kClaimsNone;
     // row entries per thread: k <= 4 * T by construction (create refuses other shapes for this block size)
     constexpr int KPT = 4;
     int32_t pos[KPT], cls[KPT];
     if (!LOOP && k <= 2 * T) {
       int32_t pos2[2], cls2[2];
-      lookup_phase<T, 2>(d, v, q, c, (uint32_t)(it & 1), stamps, pos2, cls2, my_status, any_miss, t, order_t);
+      lookup_phase<T, 2>(d, v, q, c, (uint32_t)(it & 1), stamps, pos2, cls2, my_status, any_miss, t, order_t, claims);
       if (any_miss || d.order_t == nullptr) {
-        miss_path<T, 2>(d, c, pos2, cls2, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+        miss_path<T, 2>(d, c, claims, pos2, cls2, t, order_t, my_status, fetch_parity, order_parity, gave_up);
         continue;
       }
     } else {
-      lookup_phase<T, KPT>(d, v, q, c, (uint32_t)(it & 1), stamps, pos, cls, my_status, any_miss, t, order_t);
+      lookup_phase<T, KPT>(d, v, q, c, (uint32_t)(it & 1), stamps, pos, cls, my_status, any_miss, t, order_t, claims);
       if (any_miss || d.order_t == nullptr) {
         if (LOOP) {
           // stash the thread's missing positions for the out-of-line path
@@ -1305,7 +1369,7 @@ resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_
             }
           }
         } else {
-          miss_path<T, KPT>(d, c, pos, cls, t, order_t, my_status, fetch_parity, order_parity, gave_up);
+          miss_path<T, KPT>(d, c, claims, pos, cls, t, order_t, my_status, fetch_parity, order_parity, gave_up);
         }
         continue;
       }

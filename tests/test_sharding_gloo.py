@@ -83,3 +83,64 @@ def test_two_ranks_shard_requests_and_aggregate():
     assert agg[1] == 2.0                         # max over ranks
     assert agg[2] == total_ref and agg[3] == miss_ref
     assert total_ref == STEPS * 5 * 2 * 2048
+
+
+def _oracle_selections(bench, args, rank):
+    """What rank `rank` of bench.py's multi-rank job resolves: its own workload (bench.make_workload), by the oracle."""
+    from oracle import Oracle, FLAG_NO_BYTES
+    from paper_2608_07009_b200 import inputs
+    w = bench.make_workload(args, rank, steps=args.steps + 1)
+    orc = Oracle(w.num_requests, w.num_layers, w.layers_per_group, w.cache_slots, w.top_k, w.entry_bytes, w.capacity,
+                 w.init_len, None, FLAG_NO_BYTES)
+    tr = inputs.Trace(w)
+    n, first = 0, None
+    for _ in range(args.steps):
+        sel, appended, _ = tr.step()
+        if first is None:
+            first = [int(x) for x in sel[0][0][:4]]
+        if appended:
+            orc.append()
+        for layer in range(w.num_layers):
+            _, h, m = orc.resolve(layer, sel[layer // w.layers_per_group])
+            n += int(h.sum()) + int(m.sum())
+    tr.close()
+    orc.close()
+    return n, first
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` without a launcher must start two ranks itself (never run one rank in their place): here
+    with the oracle as the per-rank worker and gloo in place of NCCL, through the same make_workload / aggregate
+    calls as the GPU arm."""
+    import json
+    import subprocess
+    sys.path.insert(0, ROOT)
+    import bench
+    argv = ["--impl", "sharding-dry-run", "--gpus", "2", "--workload", "c2", "--requests", "3", "--layers", "2",
+            "--context", "2000", "--steps", "3"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py")] + argv, env=env, capture_output=True, text=True,
+                         timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([ln for ln in out.stdout.splitlines() if ln.startswith("{")][-1])
+    args = bench.parse_args(argv)
+    want = [_oracle_selections(bench, args, r) for r in range(2)]
+    assert line["n_gpus"] == 2
+    assert line["selections"] == want[0][0] + want[1][0] and line["selections_rank0"] == want[0][0]
+    assert line["first_rows"] == [want[0][1], want[1][1]] and want[0][1] != want[1][1]   # every rank serves its own requests
+    assert line["config"]["num_requests"] == 3 and line["config"]["num_layers"] == 2
+
+
+def test_bench_refuses_more_gpus_than_there_are():
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "64", "--steps", "1"], env=env,
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode != 0 and "--gpus 64" in out.stderr and not out.stdout.strip()
+
+
+def test_cpu_list_parsing_for_numa_binding():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.parse_cpulist("0-3,8,10-11\n") == {0, 1, 2, 3, 8, 10, 11}
+    assert bench.parse_cpulist("") == set()
