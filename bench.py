@@ -123,16 +123,28 @@ def spawn_ranks(args, argv) -> int:
 
 
 def gpu_numa_node(index: int):
-    """NUMA node of the PCIe root the GPU hangs off (None when the platform does not say)."""
+    """(NUMA node of the PCIe root the GPU hangs off, or None; how it was found / why not)."""
+    bdf = None
     try:
         import torch
         p = torch.cuda.get_device_properties(index)
         bdf = "%04x:%02x:%02x.0" % (p.pci_domain_id, p.pci_bus_id, p.pci_device_id)
+    except Exception:
+        try:      # read-only query
+            out = subprocess.run(["nvidia-smi", "-i", str(index), "--query-gpu=pci.bus_id", "--format=csv,noheader"],
+                                 capture_output=True, text=True, timeout=20).stdout.strip().lower()
+            if out:
+                bdf = out[-12:] if len(out) >= 12 else out       # nvidia-smi prints an 8-digit domain
+        except Exception:
+            pass
+    if not bdf:
+        return None, "PCI address of the GPU not available"
+    try:
         with open("/sys/bus/pci/devices/%s/numa_node" % bdf) as f:
             node = int(f.read().strip())
-        return node if node >= 0 else None
     except Exception:
-        return None
+        return None, "no /sys/bus/pci/devices/%s/numa_node in this container" % bdf
+    return (node, "sysfs numa_node of %s" % bdf) if node >= 0 else (None, "the platform reports no NUMA node for %s" % bdf)
 
 
 def parse_cpulist(text: str):
@@ -148,8 +160,8 @@ def parse_cpulist(text: str):
 def bind_near_gpu(index: int) -> dict:
     """Runs this rank's threads on the CPUs of the GPU's NUMA node, so that the pinned histories it allocates next
     (first touch) and the threads that fill them are local to the GPU's PCIe root.  Returns what was done."""
-    node = gpu_numa_node(index)
-    info = {"numa_node": node, "bound": False}
+    node, how = gpu_numa_node(index)
+    info = {"numa_node": node, "bound": False, "how": how}
     if node is None:
         return info
     try:
@@ -476,17 +488,17 @@ def all_hit_points(dev, peak, sm_count):
     t_s, t_s_min, geo, n_s = one(8192, steady)
     t_f, t_f_min, _, n_f = one(2048, flushed)
     ach = ALGO_BYTES_PER_HIT * n_s / t_s / 1e9
-    traffic, commit = profile_figure("resolve_kernel_all_hit.md", "dram_bytes_per_request")
+    traffic, commit = profile_figure("resolve_kernel_all_hit.md", "dram_bytes_per_launch")
     res = {"bound": "hbm", "achieved": ach, "peak": peak["value"], "unit": "GB/s", "frac": ach / peak["value"],
            "peak_source": peak["source"], "kernel": "resolve_kernel (looping narrow blocks)",
            "workload": "scaled all-hit point: 8192 requests x 1 layer, k=2048, B=4096, every selection hits; 20 launches "
                        "back to back per timing, no flush: a launch touches ~390 MB (3x L2), so its inputs are not cached",
            "algorithmic_bytes_per_launch": ALGO_BYTES_PER_HIT * n_s, "launch_us": t_s * 1e6,
            "selections_per_s": n_s / t_s, "launch_geometry": geo,
-           "traffic": traffic * 8192 if traffic else None,
-           "traffic_source": "profiles/resolve_kernel_all_hit.md: dram__bytes_read + dram__bytes_write per request of a "
-                             "2048-request launch, scaled by the requests of this launch (commit %s)" % commit,
-           "frac_dram_bytes": (traffic * 8192 / t_s / 1e9 / peak["value"]) if traffic else None,
+           "traffic": traffic,
+           "traffic_source": "profiles/resolve_kernel_all_hit.md: dram__bytes_read + dram__bytes_write of one launch of "
+                             "this shape (commit %s)" % commit,
+           "frac_dram_bytes": (traffic / t_s / 1e9 / peak["value"]) if traffic else None,
            "flushed_2048": {"launch_us": t_f * 1e6, "launch_us_min": t_f_min * 1e6,
                             "achieved": ALGO_BYTES_PER_HIT * n_f / t_f / 1e9,
                             "frac": ALGO_BYTES_PER_HIT * n_f / t_f / 1e9 / peak["value"],

@@ -63,8 +63,9 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
                                              (hisparse_order_lag).  Results are the same either way            */
 
 #define HISPARSE_FLAG_WIDE_BLOCKS 64u       /* always one 1024-thread block per SM.  By default a handle whose grid
-                                             takes several waves (more blocks than SMs) runs two 512-thread blocks
-                                             per SM when B <= 8192 and k <= 2048 (hisparse_launch_geometry)       */
+                                             would take several waves (more blocks than SMs) runs ONE resident wave
+                                             of 512-thread blocks, three or two per SM, that loop over the requests,
+                                             when B <= 8192 and k <= 2048 (hisparse_launch_geometry)              */
 
 #define HISPARSE_FLAG_NARROW_BLOCKS 128u    /* always 512-thread blocks; EINVAL when the shape does not allow them
                                              (or together with WIDE_BLOCKS).  Results do not depend on the block size */
