@@ -183,6 +183,29 @@ int hisparse_join(hisparse_t *h, void *stream);
  * gathers from with the slot table).  Valid until destroy. */
 const void *hisparse_layer_pool(const hisparse_t *h, int layer);
 
+/* The sparse-attention consumer of the slot table (Sec. 2.1: attention is exact over the selected set; Sec. 3.4
+ * Phase 5: the attention kernel takes the selected records out of the GPU cache through the emitted slots), for
+ * records laid out as the DSA configurations have them: E = 2 D bytes = D bf16 numbers, the key of a record being all
+ * D of them and its value the first value_dims (the absorbed form of multi-head latent attention; D = 576,
+ * value_dims = 512 for a 512-number latent followed by a 64-number rotary key).  For every request n and head h
+ *     out[n][h][:] = sum_j softmax_j(scale * q[n][h][:] . rec[n][j]) * rec[n][j][:value_dims],
+ *     lse[n][h]    = log sum_j exp(scale * q[n][h][:] . rec[n][j])
+ * over the entries j of slot_table_dev [N][k] (as hisparse_resolve emits it for `layer`) that are >= 0; a row with no
+ * valid entry gives out = 0, lse = -inf.
+ *   q_dev      bf16  [N][num_heads][D], 16-byte aligned; num_heads a multiple of 16
+ *   out_dev    float [N][num_heads][value_dims]; lse_dev float [N][num_heads]
+ *   value_dims 64, 128, 256 or 512, at most D; E a multiple of 32
+ *   workspace_dev  device scratch of at least hisparse_attention_workspace_bytes bytes (the partial results of the
+ *                  blocks that share one row), caller-owned so that the call allocates nothing; 16-byte aligned
+ * Arithmetic: bf16 products accumulated in fp32 on the tensor cores, softmax weights rounded to bf16 before they
+ * multiply the values: out is within 1e-2 * max |value| of the exact result (tests/test_gpu_attention.py).
+ * Enqueues two kernels on `stream` after joining the library's side streams; capturable.  EINVAL for shapes the kernel
+ * does not take. */
+int hisparse_attention_workspace_bytes(const hisparse_t *h, int num_heads, int value_dims, size_t *bytes);
+int hisparse_sparse_attention(hisparse_t *h, int layer, const void *q_dev, int num_heads, int value_dims,
+                              const int32_t *slot_table_dev, float scale, float *out_dev, float *lse_dev,
+                              void *workspace_dev, size_t workspace_bytes, void *stream);
+
 /* Stand-in for the sparse-attention consumer, which takes the selected records out of the GPU cache through
  * the slot table (Sec. 3.4 Phase 5): copies the record of every table entry into
  * out_dev, uint8 [N][k][E], 16-byte aligned (EINVAL otherwise); entries with table value -1 are zero-filled. */

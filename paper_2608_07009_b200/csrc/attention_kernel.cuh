@@ -1,0 +1,251 @@
+// Included by hisparse.cu: the sparse-attention consumer of the slot table (Sec. 3.4 Phase 5: the attention kernel
+// reads the selected records out of the GPU cache through the emitted slots; Sec. 2.1: attention is exact over the
+// selected set).  Decode attention in the absorbed form of multi-head latent attention, the record layout of the DSA
+// configurations: a record is D bf16 numbers (E = 2 D bytes), its key all D of them, its value the first Dv.
+//
+//   out[n, h, :] = sum_j softmax_j(scale * q[n, h, :] . rec[n, j]) * rec[n, j][:Dv]      over table[n, j] >= 0
+//
+// This IS a dense contraction (a [16 heads x D] query block against the gathered records), so it runs on the tensor
+// cores (mma.sync m16n8k16, bf16 inputs, fp32 accumulation); but at 16 heads per GPU it moves 1152 bytes per record
+// for 35 KFLOP, far below the machine's ridge, so the design is the one for an HBM-bound kernel: records are gathered
+// by bulk copies (cp.async.bulk, one per record, mbarrier completion) into a double-buffered shared-memory tile while
+// the previous tile is multiplied, the selection is split over enough thread blocks to fill the GPU in one wave, two
+// blocks per SM, and a second small kernel combines the splits.
+//
+// Block = 4 warps, one request, one group of 16 heads, one contiguous split of the row's k entries, tiles of 32
+// records.  Per tile: S = Q K^T (warp w: records 8w .. 8w+7, 36 k-steps for D = 576), running row maximum across
+// the warps through shared memory, P = exp(S - m) rounded to bf16 into shared memory, O = alpha O + P V (warp w: value
+// dims [Dv/4 w, Dv/4 (w+1)), fp32 accumulators in registers).  Rows of the tile are padded by 16 bytes in shared memory,
+// which makes every ldmatrix phase hit 8 different bank groups (a 1152-byte stride would put all rows on one).
+
+namespace {
+
+constexpr int kAttTile = 32;        // records per tile
+constexpr int kAttWarps = 4;
+constexpr int kAttThreads = kAttWarps * 32;
+constexpr int kAttHeads = 16;       // heads per block (one m16 row block)
+constexpr int kAttPad = 16;         // bytes of padding per staged row
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// Partial result of one (request, head, split): Dv unnormalised output numbers, then the running maximum and the sum.
+// NV = Dv / 32 = 8-wide output tiles per warp (Dv = 512 -> 16).
+template <int NV>
+__global__ void __launch_bounds__(kAttThreads, 2)
+sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const int32_t *__restrict__ table, const int k,
+                        const __nv_bfloat16 *__restrict__ q, const int H, const float scale_log2e, const int splits,
+                        float *__restrict__ partial, uint32_t *status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int Dv = NV * 8 * kAttWarps;
+  const int D = (int)(E / 2);
+  const int row_bytes = (int)E + kAttPad;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = blockIdx.x / splits, split = blockIdx.x - n * splits, hg = blockIdx.y;
+  // this split's entries of the row: [lo, hi), whole tiles except for the row's end
+  const int per = ((k + splits - 1) / splits + kAttTile - 1) / kAttTile * kAttTile;
+  const int lo = split * per, hi = lo + per < k ? lo + per : k;
+  const int ntiles = hi > lo ? (hi - lo + kAttTile - 1) / kAttTile : 0;
+
+  unsigned char *s_q = smem_raw;                                         // [16][row_bytes]
+  unsigned char *s_kv = s_q + kAttHeads * row_bytes;                     // [2][kAttTile][row_bytes]
+  unsigned char *s_p = s_kv + 2 * kAttTile * row_bytes;                  // [16][kAttTile * 2 + 16] bf16 weights
+  float *s_red = reinterpret_cast<float *>(s_p + kAttHeads * (kAttTile * 2 + kAttPad));   // [kAttWarps][16]
+  unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_red + kAttWarps * 16);   // [2]
+  constexpr int p_stride = kAttTile * 2 + kAttPad;
+
+  if (tid < 2) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(s_bar + tid)), "r"(kAttTile) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  // the query block of this head group: 16 rows of D bf16, padded
+  {
+    const uint4 *src = reinterpret_cast<const uint4 *>(q + ((int64_t)n * H + (int64_t)hg * kAttHeads) * D);
+    const int per_row = (int)(E / 16);
+    for (int i = tid; i < kAttHeads * per_row; i += kAttThreads) {
+      const int r = i / per_row, c = i - r * per_row;
+      *reinterpret_cast<uint4 *>(s_q + r * row_bytes + c * 16) = src[i];
+    }
+  }
+  __syncthreads();
+
+  // Gather of tile t into buffer t & 1: thread j < kAttTile brings record j.  A valid entry is one bulk copy; padding
+  // (or an entry past the split's end) is zero-filled by plain stores, so that 0 weight times the row is 0, not NaN.
+  auto gather = [&](const int t) {
+    if (tid >= kAttTile) return;
+    const int j = lo + t * kAttTile + tid;
+    const int32_t rec = j < hi ? table[(int64_t)n * k + j] : -1;
+    unsigned char *dst = s_kv + ((t & 1) * kAttTile + tid) * row_bytes;
+    const uint32_t bar = smem_u32(s_bar + (t & 1));
+    if (rec >= 0) {
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)E) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(dst)), "l"(pool + (int64_t)rec * E), "r"((uint32_t)E), "r"(bar) : "memory");
+    } else {
+      for (int o = 0; o < (int)E; o += 16) *reinterpret_cast<uint4 *>(dst + o) = make_uint4(0, 0, 0, 0);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // a later tile's bulk copy writes the same bytes
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+    }
+  };
+  if (ntiles > 0) gather(0);
+  if (ntiles > 1) gather(1);
+
+  const int r0 = lane >> 2;                 // this thread's accumulator rows are r0 and r0 + 8
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float acc[NV][4];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+  bool timed_out = false;
+
+  for (int t = 0; t < ntiles; ++t) {
+    if (!mbar_wait_bounded(smem_u32(s_bar + (t & 1)), (uint32_t)((t >> 1) & 1))) timed_out = true;
+    const unsigned char *kv = s_kv + (t & 1) * kAttTile * row_bytes;
+    // S = Q K^T for this warp's 8 records: 16 x 8, k-steps of 16 over D
+    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    {
+      const uint32_t a_addr = smem_u32(s_q) + (uint32_t)((lane & 15) * row_bytes + (lane >> 4) * 16);
+      const uint32_t b_addr = smem_u32(kv) + (uint32_t)((warp * 8 + (lane & 7)) * row_bytes + (lane >> 3) * 16);
+      for (int d0 = 0; d0 < D; d0 += 32) {       // two k-steps per iteration (one ldmatrix.x4 of B)
+        uint32_t a0[4], a1[4], b[4];
+        ldsm_x4(b, b_addr + (uint32_t)d0 * 2u);
+        ldsm_x4(a0, a_addr + (uint32_t)d0 * 2u);
+        mma_bf16(sc, a0, b[0], b[1]);
+        if (d0 + 16 < D) {
+          ldsm_x4(a1, a_addr + (uint32_t)(d0 + 16) * 2u);
+          mma_bf16(sc, a1, b[2], b[3]);
+        }
+      }
+    }
+    // mask padding, scale into the base-2 domain, row maxima over the tile
+    const int jbase = lo + t * kAttTile + warp * 8 + 2 * (lane & 3);
+    float s2[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int j = jbase + (i & 1);
+      const bool valid = j < hi && table[(int64_t)n * k + j] >= 0;
+      s2[i] = valid ? sc[i] * scale_log2e : -INFINITY;
+    }
+    float mx[2] = {fmaxf(s2[0], s2[1]), fmaxf(s2[2], s2[3])};
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
+      mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
+    }
+    if ((lane & 3) == 0) { s_red[warp * 16 + r0] = mx[0]; s_red[warp * 16 + r0 + 8] = mx[1]; }
+    __syncthreads();
+    float alpha[2], m_use[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int row = r0 + 8 * i;
+      float mt = s_red[row];
+#pragma unroll
+      for (int w = 1; w < kAttWarps; ++w) mt = fmaxf(mt, s_red[w * 16 + row]);
+      const float m_new = fmaxf(m_run[i], mt);
+      alpha[i] = m_run[i] == -INFINITY ? 0.f : exp2f(m_run[i] - m_new);
+      m_use[i] = m_new == -INFINITY ? 0.f : m_new;     // a row that is all padding so far: weights 0, no NaN
+      m_run[i] = m_new;
+    }
+    float pr[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pr[i] = exp2f(s2[i] - m_use[i >> 1]);
+    l_run[0] = l_run[0] * alpha[0] + pr[0] + pr[1];
+    l_run[1] = l_run[1] * alpha[1] + pr[2] + pr[3];
+    // the weights as bf16, where every warp can read them as the A operand of P V
+    {
+      const int col = warp * 8 + 2 * (lane & 3);
+      *reinterpret_cast<uint32_t *>(s_p + r0 * p_stride + col * 2) = pack_bf16(pr[0], pr[1]);
+      *reinterpret_cast<uint32_t *>(s_p + (r0 + 8) * p_stride + col * 2) = pack_bf16(pr[2], pr[3]);
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) { acc[i][0] *= alpha[0]; acc[i][1] *= alpha[0]; acc[i][2] *= alpha[1]; acc[i][3] *= alpha[1]; }
+    __syncthreads();
+    // O += P V: this warp's value dims [warp * NV * 8, (warp + 1) * NV * 8), k-steps of 16 records
+    {
+      const uint32_t p_addr = smem_u32(s_p) + (uint32_t)((lane & 15) * p_stride + (lane >> 4) * 16);
+      const uint32_t v_addr = smem_u32(kv) + (uint32_t)(((lane & 7) + ((lane >> 3) & 1) * 8) * row_bytes + (lane >> 4) * 16) +
+                              (uint32_t)(warp * NV * 16);
+#pragma unroll
+      for (int ks = 0; ks < kAttTile / 16; ++ks) {
+        uint32_t a[4];
+        ldsm_x4(a, p_addr + (uint32_t)ks * 32u);
+#pragma unroll
+        for (int nt = 0; nt < NV; nt += 2) {
+          uint32_t b[4];
+          ldsm_x4_trans(b, v_addr + (uint32_t)(ks * 16 * row_bytes) + (uint32_t)nt * 16u);
+          mma_bf16(acc[nt], a, b[0], b[1]);
+          mma_bf16(acc[nt + 1], a, b[2], b[3]);
+        }
+      }
+    }
+    __syncthreads();   // every warp is done with this tile's buffer, the weights and the maxima
+    if (t + 2 < ntiles) gather(t + 2);
+  }
+
+  // partial sums of the weights: across the quad, then across the warps (each warp summed its own 8 columns per tile)
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
+    l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
+  }
+  if ((lane & 3) == 0) { s_red[warp * 16 + r0] = l_run[0]; s_red[warp * 16 + r0 + 8] = l_run[1]; }
+  __syncthreads();
+  float *out = partial + (((int64_t)n * H + (int64_t)hg * kAttHeads) * splits + split) * (Dv + 2);
+  const int64_t head_stride = (int64_t)splits * (Dv + 2);
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int col = warp * NV * 8 + i * 8 + 2 * (lane & 3);
+    *reinterpret_cast<float2 *>(out + (int64_t)r0 * head_stride + col) = make_float2(acc[i][0], acc[i][1]);
+    *reinterpret_cast<float2 *>(out + (int64_t)(r0 + 8) * head_stride + col) = make_float2(acc[i][2], acc[i][3]);
+  }
+  if (warp == 0 && (lane & 3) == 0) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int row = r0 + 8 * i;
+      float l = 0.f;
+#pragma unroll
+      for (int w = 0; w < kAttWarps; ++w) l += s_red[w * 16 + row];
+      out[(int64_t)row * head_stride + Dv] = m_run[i];
+      out[(int64_t)row * head_stride + Dv + 1] = l;
+    }
+  }
+  if (timed_out && tid == 0) atomicOr(status, HISPARSE_STATUS_TIMEOUT);
+}
+
+// out[n, h, :] = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,  lse = ln 2 * (M + log2 L).  One block per (n, h).
+__global__ void sparse_attention_combine_kernel(const float *__restrict__ partial, const int splits, const int Dv,
+                                                float *__restrict__ out, float *__restrict__ lse) {
+  const int64_t nh = blockIdx.x;
+  const float *p = partial + nh * splits * (Dv + 2);
+  float M = -INFINITY;
+  for (int s = 0; s < splits; ++s) M = fmaxf(M, p[(int64_t)s * (Dv + 2) + Dv]);
+  float L = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float m = p[(int64_t)s * (Dv + 2) + Dv];
+    if (m != -INFINITY) L += exp2f(m - M) * p[(int64_t)s * (Dv + 2) + Dv + 1];
+  }
+  for (int c = threadIdx.x; c < Dv; c += blockDim.x) {
+    float o = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float m = p[(int64_t)s * (Dv + 2) + Dv];
+      if (m != -INFINITY) o += exp2f(m - M) * p[(int64_t)s * (Dv + 2) + c];
+    }
+    out[nh * Dv + c] = L > 0.f ? o / L : 0.f;
+  }
+  if (threadIdx.x == 0) lse[nh] = L > 0.f ? 0.6931471805599453f * (M + log2f(L)) : -INFINITY;
+}
+
+}  // namespace

@@ -31,6 +31,7 @@
 // launched as one resident wave of 512-thread blocks (three or two per SM) that loop over the requests.
 #include "hisparse.h"
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -44,5 +45,6 @@
 #include "device_common.cuh"
 #include "resolve_kernel.cuh"
 #include "aux_kernels.cuh"
+#include "attention_kernel.cuh"
 #include "host_api.inl"
 #include "noalloc.inl"

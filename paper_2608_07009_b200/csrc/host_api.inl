@@ -149,6 +149,46 @@ int launch_replay(hisparse *h, int layer, cudaStream_t st) {
 
 }  // namespace
 
+// ---- the sparse-attention consumer (attention_kernel.cuh) ----
+
+namespace {
+
+struct AttGeom { int splits, tiles_per_split; size_t smem, workspace; };
+
+// Splits of a row's k entries such that the launch fills the GPU once at two blocks per SM, in whole tiles.
+int attention_geometry(const hisparse *h, int num_heads, int value_dims, AttGeom *g) {
+  const int64_t E = h->d.E;
+  if (num_heads < kAttHeads || num_heads % kAttHeads) return HISPARSE_EINVAL;
+  if (E % 32 || !(value_dims == 64 || value_dims == 128 || value_dims == 256 || value_dims == 512) || value_dims > E / 2)
+    return HISPARSE_EINVAL;
+  const int tiles = (h->d.k + kAttTile - 1) / kAttTile;
+  const int64_t groups = (int64_t)h->d.N * (num_heads / kAttHeads);
+  int want = (int)std::max<int64_t>(1, (2 * (int64_t)h->sm_count) / groups);
+  want = std::min(want, tiles);
+  g->tiles_per_split = (tiles + want - 1) / want;
+  g->splits = (tiles + g->tiles_per_split - 1) / g->tiles_per_split;
+  const size_t row = (size_t)E + kAttPad;
+  g->smem = kAttHeads * row + 2 * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttWarps * 16 * 4 + 16;
+  g->workspace = (size_t)h->d.N * num_heads * g->splits * (value_dims + 2) * sizeof(float);
+  return HISPARSE_OK;
+}
+
+template <int NV>
+int launch_attention(hisparse *h, const AttGeom &g, const uint8_t *pool, const int32_t *table, const __nv_bfloat16 *q,
+                     int num_heads, float scale, float *partial, cudaStream_t st) {
+  int optin = 0;
+  HS_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
+  if (g.smem > (size_t)optin) return HISPARSE_EINVAL;
+  HS_CUDA(cudaFuncSetAttribute(sparse_attention_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem));
+  const dim3 grid((unsigned)(h->d.N * g.splits), (unsigned)(num_heads / kAttHeads));
+  sparse_attention_kernel<NV><<<grid, kAttThreads, g.smem, st>>>(pool, h->d.E, table, h->d.k, q, num_heads,
+                                                                 scale * 1.4426950408889634f, g.splits, partial, h->d.status);
+  HS_CUDA(cudaGetLastError());
+  return HISPARSE_OK;
+}
+
+}  // namespace
+
 // ------------------------------------------------------------------------------------------ C-ABI
 
 extern "C" {
@@ -511,6 +551,43 @@ int hisparse_prefetch_hint(hisparse_t *h, int layer, const int32_t *hint_sel_dev
   h->anchor_done[layer] = 1;
   HS_CUDA(cudaEventRecord(h->ev_hint[layer], side));
   h->hint_unjoined[layer] = 1;
+  return HISPARSE_OK;
+}
+
+int hisparse_attention_workspace_bytes(const hisparse_t *h, int num_heads, int value_dims, size_t *bytes) {
+  if (!h || !bytes) return HISPARSE_EINVAL;
+  AttGeom g;
+  const int rc = attention_geometry(h, num_heads, value_dims, &g);
+  if (rc) return rc;
+  *bytes = g.workspace;
+  return HISPARSE_OK;
+}
+
+int hisparse_sparse_attention(hisparse_t *h, int layer, const void *q_dev, int num_heads, int value_dims,
+                              const int32_t *slot_table_dev, float scale, float *out_dev, float *lse_dev,
+                              void *workspace_dev, size_t workspace_bytes, void *stream) {
+  if (!h || layer < 0 || layer >= h->d.L || !q_dev || !slot_table_dev || !out_dev || !lse_dev || !workspace_dev)
+    return HISPARSE_EINVAL;
+  if (((uintptr_t)q_dev | (uintptr_t)workspace_dev | (uintptr_t)out_dev) & 15) return HISPARSE_EINVAL;
+  AttGeom g;
+  int rc = attention_geometry(h, num_heads, value_dims, &g);
+  if (rc) return rc;
+  if (workspace_bytes < g.workspace) return HISPARSE_EINVAL;
+  rc = hisparse_join(h, stream);   // a prefetch replay or a write-through may still be filling this layer's cache
+  if (rc) return rc;
+  cudaStream_t st = as_stream(stream);
+  const uint8_t *pool = h->d.pool + (int64_t)layer * h->d.layer_pool_bytes;
+  const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(q_dev);
+  float *partial = static_cast<float *>(workspace_dev);
+  switch (value_dims) {
+    case 64: rc = launch_attention<2>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+    case 128: rc = launch_attention<4>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+    case 256: rc = launch_attention<8>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+    default: rc = launch_attention<16>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+  }
+  if (rc) return rc;
+  sparse_attention_combine_kernel<<<(unsigned)(h->d.N * num_heads), 128, 0, st>>>(partial, g.splits, value_dims, out_dev, lse_dev);
+  HS_CUDA(cudaGetLastError());
   return HISPARSE_OK;
 }
 

@@ -28,6 +28,7 @@ EXPORTS = [
     "hisparse_clear_status", "hisparse_dump_state", "hisparse_order_lag", "hisparse_load_state", "hisparse_load_appends", "hisparse_dump_plan", "hisparse_device_bytes",
     "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_selftest_wait_timeout", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
     "hisparse_scatter_read_probe", "hisparse_resolve_noalloc", "hisparse_strerror", "hisparse_last_cuda_error",
+    "hisparse_attention_workspace_bytes", "hisparse_sparse_attention",
 ]
 
 
@@ -102,6 +103,8 @@ def lib() -> ctypes.CDLL:
             "hisparse_host_link_probe": ([i32, sz, i32, P(ctypes.c_double)], i32),
             "hisparse_scatter_read_probe": ([i32, vp, sz, i64, ctypes.c_int32, ctypes.c_int32, i32, P(ctypes.c_double)], i32),
             "hisparse_resolve_noalloc": ([P(ExternalState), vp, vp, vp, vp, vp, vp], i32),
+            "hisparse_attention_workspace_bytes": ([vp, i32, i32, P(sz)], i32),
+            "hisparse_sparse_attention": ([vp, i32, vp, i32, i32, vp, ctypes.c_float, vp, vp, vp, sz, vp], i32),
             "hisparse_strerror": ([i32], ctypes.c_char_p),
             "hisparse_last_cuda_error": ([], i32),
         }
@@ -258,6 +261,36 @@ class HiSparse:
 
     def join(self, stream=None) -> None:
         _check(lib().hisparse_join(self._h, _stream_ptr(stream)), "hisparse_join")
+
+    # ---- the sparse-attention consumer ----
+    def attention_workspace_bytes(self, num_heads: int, value_dims: int) -> int:
+        n = ctypes.c_size_t()
+        _check(lib().hisparse_attention_workspace_bytes(self._h, num_heads, value_dims, ctypes.byref(n)),
+               "hisparse_attention_workspace_bytes")
+        return n.value
+
+    def sparse_attention(self, layer: int, q, slot_table, value_dims: int, scale: float, out=None, lse=None,
+                         workspace=None, stream=None):
+        """q: bf16 CUDA tensor [N][H][E/2]; returns (out float32 [N][H][value_dims], lse float32 [N][H])."""
+        import torch
+        dev = "cuda:%d" % self.device
+        H = q.shape[1]
+        if not (q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous() and q.shape == (self.N, H, self.E // 2)):
+            raise ValueError("expected a contiguous CUDA bfloat16 tensor [N][H][E/2]")
+        if out is None:
+            out = torch.empty((self.N, H, value_dims), dtype=torch.float32, device=dev)
+        if lse is None:
+            lse = torch.empty((self.N, H), dtype=torch.float32, device=dev)
+        need = self.attention_workspace_bytes(H, value_dims)
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+        _check(lib().hisparse_sparse_attention(self._h, layer, q.data_ptr(), H, value_dims,
+                                               _dev_ptr(slot_table, "int32", self.N * self.k), scale,
+                                               _dev_ptr(out, "float32", self.N * H * value_dims),
+                                               _dev_ptr(lse, "float32", self.N * H), workspace.data_ptr(),
+                                               workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+               "hisparse_sparse_attention")
+        return out, lse
 
     # ---- consumer stand-ins ----
     def layer_pool(self, layer: int) -> int:
