@@ -769,6 +769,37 @@ def measure(args, w, dev, local, K, W, full, launched, rank):
                                "hbm_gb_s": 2 * N * k * E / t_g / 1e9,
                                "frac_of_hbm_peak": 2 * N * k * E / t_g / 1e9 / peak["value"], "peak_source": peak["source"]}
             del out_buf
+    # ---- the real consumer: sparse decode attention over the selected records (16 heads, MLA record layout) ----
+    out["attention"] = None
+    if full and not args.skip_io and E == 1152:
+        with torch.cuda.stream(main):
+            heads, dv = 16, 512
+            q_att = torch.randn((N, heads, E // 2), device=dev).to(torch.bfloat16)
+            o_att = torch.empty((N, heads, dv), dtype=torch.float32, device=dev)
+            l_att = torch.empty((N, heads), dtype=torch.float32, device=dev)
+            ws = torch.empty(gpu.attention_workspace_bytes(heads, dv), dtype=torch.uint8, device=dev)
+            ts = []
+            for i in range(3 + 8):
+                flush()
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(main)
+                gpu.sparse_attention(0, q_att, tabs[0], dv, (E // 2) ** -0.5, o_att, l_att, ws, stream=main)
+                b_.record(main)
+                b_.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b_) * 1e-3)
+            t_a = statistics.mean(ts)
+            valid = int((tabs[0] >= 0).sum().item())
+            nbytes = valid * E + q_att.numel() * 2 + o_att.numel() * 4
+            flops = 2.0 * heads * valid * (E // 2 + dv)
+            peak = hbm_peak()
+            out["attention"] = {"kernel": "sparse_attention_kernel + combine", "heads": heads, "value_dims": dv,
+                                "launch_us": t_a * 1e6, "algorithmic_bytes": nbytes, "hbm_gb_s": nbytes / t_a / 1e9,
+                                "frac_of_hbm_peak": nbytes / t_a / 1e9 / peak["value"], "peak_source": peak["source"],
+                                "tflops": flops / t_a / 1e12,
+                                "note": "layer 0's table of the last step; each selected record read once; L2 flushed "
+                                        "between launches"}
+            del q_att, o_att, l_att, ws
     out["status"] = status | gpu.status()
     out["sm_read"] = None
     if full:
@@ -918,6 +949,7 @@ def run_ours(args):
                       "note": "copy-only kernel, one block per SM, random records of this workload's size"},
         "placement": placement,
         "cold_step_ms": m["cold_ms"], "hit_only_step": m["hit_only"], "consumer_gather": m["consumer"],
+        "consumer_attention": m["attention"],
         "status_bits": m["status"], "launch_geometry": m["geo"], "setup_s": m["setup_s"], "pinned_bytes": m["pinned_bytes"],
     }
     if "phases" in m:

@@ -68,10 +68,14 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   unsigned char *s_p = s_kv + 2 * kAttTile * row_bytes;                  // [16][kAttTile * 2 + 16] bf16 weights
   float *s_red = reinterpret_cast<float *>(s_p + kAttHeads * (kAttTile * 2 + kAttPad));   // [kAttWarps][16]
   unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_red + kAttWarps * 16);   // [2]
+  int32_t *s_tab = reinterpret_cast<int32_t *>(s_bar + 2);               // [per]: this split's table entries
   constexpr int p_stride = kAttTile * 2 + kAttPad;
 
   if (tid < 2) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(s_bar + tid)), "r"(kAttTile) : "memory");
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  // this split's slice of the row (-1 past its end): read once, so that neither the gather nor the masking waits
+  // for global memory inside the tile loop
+  for (int i = tid; i < per; i += kAttThreads) s_tab[i] = lo + i < hi ? table[(int64_t)n * k + lo + i] : -1;
   // the query block of this head group: 16 rows of D bf16, padded
   {
     const uint4 *src = reinterpret_cast<const uint4 *>(q + ((int64_t)n * H + (int64_t)hg * kAttHeads) * D);
@@ -87,8 +91,7 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   // (or an entry past the split's end) is zero-filled by plain stores, so that 0 weight times the row is 0, not NaN.
   auto gather = [&](const int t) {
     if (tid >= kAttTile) return;
-    const int j = lo + t * kAttTile + tid;
-    const int32_t rec = j < hi ? table[(int64_t)n * k + j] : -1;
+    const int32_t rec = s_tab[t * kAttTile + tid];
     unsigned char *dst = s_kv + ((t & 1) * kAttTile + tid) * row_bytes;
     const uint32_t bar = smem_u32(s_bar + (t & 1));
     if (rec >= 0) {
@@ -115,30 +118,41 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
     if (!mbar_wait_bounded(smem_u32(s_bar + (t & 1)), (uint32_t)((t >> 1) & 1))) timed_out = true;
     const unsigned char *kv = s_kv + (t & 1) * kAttTile * row_bytes;
     // S = Q K^T for this warp's 8 records: 16 x 8, k-steps of 16 over D
-    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    // (four independent accumulators, summed at the end: one accumulator would make the 36 MMAs one dependent chain)
+    float sc[4];
     {
+      float part[4][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) part[i][0] = part[i][1] = part[i][2] = part[i][3] = 0.f;
       const uint32_t a_addr = smem_u32(s_q) + (uint32_t)((lane & 15) * row_bytes + (lane >> 4) * 16);
       const uint32_t b_addr = smem_u32(kv) + (uint32_t)((warp * 8 + (lane & 7)) * row_bytes + (lane >> 3) * 16);
-      for (int d0 = 0; d0 < D; d0 += 32) {       // two k-steps per iteration (one ldmatrix.x4 of B)
-        uint32_t a0[4], a1[4], b[4];
-        ldsm_x4(b, b_addr + (uint32_t)d0 * 2u);
-        ldsm_x4(a0, a_addr + (uint32_t)d0 * 2u);
-        mma_bf16(sc, a0, b[0], b[1]);
-        if (d0 + 16 < D) {
-          ldsm_x4(a1, a_addr + (uint32_t)(d0 + 16) * 2u);
-          mma_bf16(sc, a1, b[2], b[3]);
-        }
+      int d0 = 0;
+#pragma unroll 3
+      for (; d0 + 64 <= D; d0 += 64) {           // four k-steps per iteration (two ldmatrix.x4 of B)
+        uint32_t a[4][4], b0[4], b1[4];
+        ldsm_x4(b0, b_addr + (uint32_t)d0 * 2u);
+        ldsm_x4(b1, b_addr + (uint32_t)(d0 + 32) * 2u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ldsm_x4(a[i], a_addr + (uint32_t)(d0 + 16 * i) * 2u);
+        mma_bf16(part[0], a[0], b0[0], b0[1]);
+        mma_bf16(part[1], a[1], b0[2], b0[3]);
+        mma_bf16(part[2], a[2], b1[0], b1[1]);
+        mma_bf16(part[3], a[3], b1[2], b1[3]);
       }
+      for (; d0 < D; d0 += 16) {                 // what is left of D (a multiple of 16)
+        uint32_t a[4], b[4];
+        ldsm_x4(b, b_addr + (uint32_t)d0 * 2u);   // its upper half may lie past the row's end: not used
+        ldsm_x4(a, a_addr + (uint32_t)d0 * 2u);
+        mma_bf16(part[0], a, b[0], b[1]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) sc[i] = (part[0][i] + part[1][i]) + (part[2][i] + part[3][i]);
     }
     // mask padding, scale into the base-2 domain, row maxima over the tile
-    const int jbase = lo + t * kAttTile + warp * 8 + 2 * (lane & 3);
+    const int jbase = t * kAttTile + warp * 8 + 2 * (lane & 3);
     float s2[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int j = jbase + (i & 1);
-      const bool valid = j < hi && table[(int64_t)n * k + j] >= 0;
-      s2[i] = valid ? sc[i] * scale_log2e : -INFINITY;
-    }
+    for (int i = 0; i < 4; ++i) s2[i] = s_tab[jbase + (i & 1)] >= 0 ? sc[i] * scale_log2e : -INFINITY;
     float mx[2] = {fmaxf(s2[0], s2[1]), fmaxf(s2[2], s2[3])};
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
@@ -170,8 +184,10 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       *reinterpret_cast<uint32_t *>(s_p + r0 * p_stride + col * 2) = pack_bf16(pr[0], pr[1]);
       *reinterpret_cast<uint32_t *>(s_p + (r0 + 8) * p_stride + col * 2) = pack_bf16(pr[2], pr[3]);
     }
+    if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {   // (a maximum moved: rescale what was summed so far)
 #pragma unroll
-    for (int i = 0; i < NV; ++i) { acc[i][0] *= alpha[0]; acc[i][1] *= alpha[0]; acc[i][2] *= alpha[1]; acc[i][3] *= alpha[1]; }
+      for (int i = 0; i < NV; ++i) { acc[i][0] *= alpha[0]; acc[i][1] *= alpha[0]; acc[i][2] *= alpha[1]; acc[i][3] *= alpha[1]; }
+    }
     __syncthreads();
     // O += P V: this warp's value dims [warp * NV * 8, (warp + 1) * NV * 8), k-steps of 16 records
     {

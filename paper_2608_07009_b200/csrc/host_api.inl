@@ -168,7 +168,8 @@ int attention_geometry(const hisparse *h, int num_heads, int value_dims, AttGeom
   g->tiles_per_split = (tiles + want - 1) / want;
   g->splits = (tiles + g->tiles_per_split - 1) / g->tiles_per_split;
   const size_t row = (size_t)E + kAttPad;
-  g->smem = kAttHeads * row + 2 * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttWarps * 16 * 4 + 16;
+  g->smem = kAttHeads * row + 2 * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttWarps * 16 * 4 + 16 +
+            (size_t)g->tiles_per_split * kAttTile * 4;
   g->workspace = (size_t)h->d.N * num_heads * g->splits * (value_dims + 2) * sizeof(float);
   return HISPARSE_OK;
 }
