@@ -12,16 +12,19 @@
 // the previous tile is multiplied, the selection is split over enough thread blocks to fill the GPU in one wave, two
 // blocks per SM, and a second small kernel combines the splits.
 //
-// Block = 4 warps, one request, one group of 16 heads, one contiguous split of the row's k entries, tiles of 32
-// records.  Per tile: S = Q K^T (warp w: records 8w .. 8w+7, 36 k-steps for D = 576), running row maximum across
-// the warps through shared memory, P = exp(S - m) rounded to bf16 into shared memory, O = alpha O + P V (warp w: value
-// dims [Dv/4 w, Dv/4 (w+1)), fp32 accumulators in registers).  Rows of the tile are padded by 16 bytes in shared memory,
+// Block = 8 warps, one request, one group of 16 heads, one contiguous split of the row's k entries, tiles of 32
+// records.  Per tile: S = Q K^T (warp w: records 8 (w & 3) .. + 7 over one half of D, the two halves added through
+// shared memory), running row maximum across the record groups through shared memory, P = exp(S - m) rounded to
+// bf16 into shared memory, O = alpha O + P V (warp w: value dims [Dv/8 w, Dv/8 (w+1)), fp32 accumulators in
+// registers).  Eight warps rather than four: a tile is a serial chain of ldmatrix -> mma -> maximum -> exp -> mma with
+// block barriers in between, and with 8 warps per SM the schedulers issued on 17 % of their cycles.  Rows of the tile are padded by 16 bytes in shared memory,
 // which makes every ldmatrix phase hit 8 different bank groups (a 1152-byte stride would put all rows on one).
 
 namespace {
 
 constexpr int kAttTile = 32;        // records per tile
-constexpr int kAttWarps = 4;
+constexpr int kAttWarps = 8;
+constexpr int kAttGroups = kAttTile / 8;   // groups of 8 records (one n-tile of the score MMA) per tile
 constexpr int kAttThreads = kAttWarps * 32;
 constexpr int kAttHeads = 16;       // heads per block (one m16 row block)
 constexpr int kAttPad = 16;         // bytes of padding per staged row
@@ -45,8 +48,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-// Partial result of one (request, head, split): Dv unnormalised output numbers, then the running maximum and the sum.
-// NV = Dv / 32 = 8-wide output tiles per warp (Dv = 512 -> 16).
+// Partial result of one (request, head, split): Dv unnormalised output numbers, then the running maximum (base 2) and
+// the sum of the weights, padded to Dv + 4 floats so that rows stay 16-byte aligned.
+// NV = Dv / 64 = 8-wide output tiles per warp (Dv = 512 -> 8).
 template <int NV>
 __global__ void __launch_bounds__(kAttThreads, 2)
 sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const int32_t *__restrict__ table, const int k,
@@ -66,8 +70,9 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   unsigned char *s_q = smem_raw;                                         // [16][row_bytes]
   unsigned char *s_kv = s_q + kAttHeads * row_bytes;                     // [2][kAttTile][row_bytes]
   unsigned char *s_p = s_kv + 2 * kAttTile * row_bytes;                  // [16][kAttTile * 2 + 16] bf16 weights
-  float *s_red = reinterpret_cast<float *>(s_p + kAttHeads * (kAttTile * 2 + kAttPad));   // [kAttWarps][16]
-  unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_red + kAttWarps * 16);   // [2]
+  float *s_red = reinterpret_cast<float *>(s_p + kAttHeads * (kAttTile * 2 + kAttPad));   // [kAttGroups][16]
+  float4 *s_part = reinterpret_cast<float4 *>(s_red + kAttGroups * 16);                    // [kAttWarps][32]: half scores
+  unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_part + kAttWarps * 32);   // [2]
   int32_t *s_tab = reinterpret_cast<int32_t *>(s_bar + 2);               // [per]: this split's table entries
   constexpr int p_stride = kAttTile * 2 + kAttPad;
 
@@ -89,8 +94,10 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
 
   // Gather of tile t into buffer t & 1: thread j < kAttTile brings record j.  A valid entry is one bulk copy; padding
   // (or an entry past the split's end) is zero-filled by plain stores, so that 0 weight times the row is 0, not NaN.
+  // (16-byte cp.async copies by all threads instead: 32.7 us against 30 us; asking the later tiles' records into L2
+  // with one prefetch each at the start: 37 us.  Both measured on the C2 shape, neither kept.)
   auto gather = [&](const int t) {
-    if (tid >= kAttTile) return;
+    if (tid >= kAttTile || t >= ntiles) return;
     const int32_t rec = s_tab[t * kAttTile + tid];
     unsigned char *dst = s_kv + ((t & 1) * kAttTile + tid) * row_bytes;
     const uint32_t bar = smem_u32(s_bar + (t & 1));
@@ -104,10 +111,13 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
     }
   };
-  if (ntiles > 0) gather(0);
-  if (ntiles > 1) gather(1);
+  gather(0);
+  gather(1);
 
   const int r0 = lane >> 2;                 // this thread's accumulator rows are r0 and r0 + 8
+  const int grp = warp & (kAttGroups - 1);  // the 8 records of a tile this warp scores ...
+  const bool half = warp >= kAttGroups;     // ... over the lower or the upper half of D
+  const int d_mid = ((D / 16 + 1) / 2) * 16, d_lo = half ? d_mid : 0, d_hi = half ? D : d_mid;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   float acc[NV][4];
 #pragma unroll
@@ -117,18 +127,18 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   for (int t = 0; t < ntiles; ++t) {
     if (!mbar_wait_bounded(smem_u32(s_bar + (t & 1)), (uint32_t)((t >> 1) & 1))) timed_out = true;
     const unsigned char *kv = s_kv + (t & 1) * kAttTile * row_bytes;
-    // S = Q K^T for this warp's 8 records: 16 x 8, k-steps of 16 over D
-    // (four independent accumulators, summed at the end: one accumulator would make the 36 MMAs one dependent chain)
+    // S = Q K^T for this warp's 8 records over its half of D: 16 x 8, k-steps of 16
+    // (four independent accumulators, summed at the end: one accumulator would make the MMAs one dependent chain)
     float sc[4];
     {
       float part[4][4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) part[i][0] = part[i][1] = part[i][2] = part[i][3] = 0.f;
       const uint32_t a_addr = smem_u32(s_q) + (uint32_t)((lane & 15) * row_bytes + (lane >> 4) * 16);
-      const uint32_t b_addr = smem_u32(kv) + (uint32_t)((warp * 8 + (lane & 7)) * row_bytes + (lane >> 3) * 16);
-      int d0 = 0;
-#pragma unroll 3
-      for (; d0 + 64 <= D; d0 += 64) {           // four k-steps per iteration (two ldmatrix.x4 of B)
+      const uint32_t b_addr = smem_u32(kv) + (uint32_t)((grp * 8 + (lane & 7)) * row_bytes + (lane >> 3) * 16);
+      int d0 = d_lo;
+#pragma unroll 2
+      for (; d0 + 64 <= d_hi; d0 += 64) {        // four k-steps per iteration (two ldmatrix.x4 of B)
         uint32_t a[4][4], b0[4], b1[4];
         ldsm_x4(b0, b_addr + (uint32_t)d0 * 2u);
         ldsm_x4(b1, b_addr + (uint32_t)(d0 + 32) * 2u);
@@ -139,17 +149,25 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
         mma_bf16(part[2], a[2], b1[0], b1[1]);
         mma_bf16(part[3], a[3], b1[2], b1[3]);
       }
-      for (; d0 < D; d0 += 16) {                 // what is left of D (a multiple of 16)
+      for (; d0 < d_hi; d0 += 16) {              // what is left of the half (a multiple of 16)
         uint32_t a[4], b[4];
         ldsm_x4(b, b_addr + (uint32_t)d0 * 2u);   // its upper half may lie past the row's end: not used
         ldsm_x4(a, a_addr + (uint32_t)d0 * 2u);
         mma_bf16(part[0], a, b[0], b[1]);
       }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) sc[i] = (part[0][i] + part[1][i]) + (part[2][i] + part[3][i]);
+      const float4 mine = make_float4((part[0][0] + part[1][0]) + (part[2][0] + part[3][0]),
+                                      (part[0][1] + part[1][1]) + (part[2][1] + part[3][1]),
+                                      (part[0][2] + part[1][2]) + (part[2][2] + part[3][2]),
+                                      (part[0][3] + part[1][3]) + (part[2][3] + part[3][3]));
+      s_part[warp * 32 + lane] = mine;
+      __syncthreads();
+      const float4 other = s_part[(warp ^ kAttGroups) * 32 + lane];   // the same records, the other half of D
+      // (added in a fixed order, so that both warps of a pair hold bit-identical scores)
+      const float4 lo4 = half ? other : mine, hi4 = half ? mine : other;
+      sc[0] = lo4.x + hi4.x; sc[1] = lo4.y + hi4.y; sc[2] = lo4.z + hi4.z; sc[3] = lo4.w + hi4.w;
     }
     // mask padding, scale into the base-2 domain, row maxima over the tile
-    const int jbase = t * kAttTile + warp * 8 + 2 * (lane & 3);
+    const int jbase = t * kAttTile + grp * 8 + 2 * (lane & 3);
     float s2[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) s2[i] = s_tab[jbase + (i & 1)] >= 0 ? sc[i] * scale_log2e : -INFINITY;
@@ -159,7 +177,7 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
       mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
     }
-    if ((lane & 3) == 0) { s_red[warp * 16 + r0] = mx[0]; s_red[warp * 16 + r0 + 8] = mx[1]; }
+    if ((lane & 3) == 0 && !half) { s_red[grp * 16 + r0] = mx[0]; s_red[grp * 16 + r0 + 8] = mx[1]; }
     __syncthreads();
     float alpha[2], m_use[2];
 #pragma unroll
@@ -167,7 +185,7 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       const int row = r0 + 8 * i;
       float mt = s_red[row];
 #pragma unroll
-      for (int w = 1; w < kAttWarps; ++w) mt = fmaxf(mt, s_red[w * 16 + row]);
+      for (int w = 1; w < kAttGroups; ++w) mt = fmaxf(mt, s_red[w * 16 + row]);
       const float m_new = fmaxf(m_run[i], mt);
       alpha[i] = m_run[i] == -INFINITY ? 0.f : exp2f(m_run[i] - m_new);
       m_use[i] = m_new == -INFINITY ? 0.f : m_new;     // a row that is all padding so far: weights 0, no NaN
@@ -179,8 +197,8 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
     l_run[0] = l_run[0] * alpha[0] + pr[0] + pr[1];
     l_run[1] = l_run[1] * alpha[1] + pr[2] + pr[3];
     // the weights as bf16, where every warp can read them as the A operand of P V
-    {
-      const int col = warp * 8 + 2 * (lane & 3);
+    if (!half) {
+      const int col = grp * 8 + 2 * (lane & 3);
       *reinterpret_cast<uint32_t *>(s_p + r0 * p_stride + col * 2) = pack_bf16(pr[0], pr[1]);
       *reinterpret_cast<uint32_t *>(s_p + (r0 + 8) * p_stride + col * 2) = pack_bf16(pr[2], pr[3]);
     }
@@ -208,19 +226,19 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       }
     }
     __syncthreads();   // every warp is done with this tile's buffer, the weights and the maxima
-    if (t + 2 < ntiles) gather(t + 2);
+    gather(t + 2);
   }
 
-  // partial sums of the weights: across the quad, then across the warps (each warp summed its own 8 columns per tile)
+  // partial sums of the weights: across the quad, then across the record groups (one warp of each pair reports)
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
     l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
   }
-  if ((lane & 3) == 0) { s_red[warp * 16 + r0] = l_run[0]; s_red[warp * 16 + r0 + 8] = l_run[1]; }
+  if ((lane & 3) == 0 && !half) { s_red[grp * 16 + r0] = l_run[0]; s_red[grp * 16 + r0 + 8] = l_run[1]; }
   __syncthreads();
-  float *out = partial + (((int64_t)n * H + (int64_t)hg * kAttHeads) * splits + split) * (Dv + 2);
-  const int64_t head_stride = (int64_t)splits * (Dv + 2);
+  float *out = partial + (((int64_t)n * H + (int64_t)hg * kAttHeads) * splits + split) * (Dv + 4);
+  const int64_t head_stride = (int64_t)splits * (Dv + 4);
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
     const int col = warp * NV * 8 + i * 8 + 2 * (lane & 3);
@@ -233,7 +251,7 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       const int row = r0 + 8 * i;
       float l = 0.f;
 #pragma unroll
-      for (int w = 0; w < kAttWarps; ++w) l += s_red[w * 16 + row];
+      for (int w = 0; w < kAttGroups; ++w) l += s_red[w * 16 + row];
       out[(int64_t)row * head_stride + Dv] = m_run[i];
       out[(int64_t)row * head_stride + Dv + 1] = l;
     }
@@ -241,27 +259,45 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   if (timed_out && tid == 0) atomicOr(status, HISPARSE_STATUS_TIMEOUT);
 }
 
-// out[n, h, :] = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,  lse = ln 2 * (M + log2 L).  One block per (n, h).
-__global__ void sparse_attention_combine_kernel(const float *__restrict__ partial, const int splits, const int Dv,
-                                                float *__restrict__ out, float *__restrict__ lse) {
+// out[n, h, :] = sum_s 2^(m_s - M) o_s / sum_s 2^(m_s - M) l_s,  lse = ln 2 * (M + log2 L).  One block of 128 threads
+// per (n, h); splits <= 128 (one per tile of a row of at most 4096 entries).
+__global__ void __launch_bounds__(128)
+sparse_attention_combine_kernel(const float *__restrict__ partial, const int splits, const int Dv,
+                                float *__restrict__ out, float *__restrict__ lse) {
+  __shared__ float s_w[128];
+  __shared__ float s_red[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t nh = blockIdx.x;
-  const float *p = partial + nh * splits * (Dv + 2);
-  float M = -INFINITY;
-  for (int s = 0; s < splits; ++s) M = fmaxf(M, p[(int64_t)s * (Dv + 2) + Dv]);
-  float L = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    const float m = p[(int64_t)s * (Dv + 2) + Dv];
-    if (m != -INFINITY) L += exp2f(m - M) * p[(int64_t)s * (Dv + 2) + Dv + 1];
-  }
-  for (int c = threadIdx.x; c < Dv; c += blockDim.x) {
-    float o = 0.f;
+  const int stride = Dv + 4;
+  const float *p = partial + nh * splits * stride;
+  const float m = tid < splits ? p[(int64_t)tid * stride + Dv] : -INFINITY;
+  const float l = tid < splits ? p[(int64_t)tid * stride + Dv + 1] : 0.f;
+  float M = m;
+#pragma unroll
+  for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  if (lane == 0) s_red[warp] = M;
+  __syncthreads();
+  M = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+  const float w = m == -INFINITY ? 0.f : exp2f(m - M);
+  s_w[tid] = w;
+  float L = w * l;
+#pragma unroll
+  for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+  if (lane == 0) s_red[4 + warp] = L;
+  __syncthreads();
+  L = (s_red[4] + s_red[5]) + (s_red[6] + s_red[7]);
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  for (int c = tid * 4; c < Dv; c += 128 * 4) {
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
     for (int s = 0; s < splits; ++s) {
-      const float m = p[(int64_t)s * (Dv + 2) + Dv];
-      if (m != -INFINITY) o += exp2f(m - M) * p[(int64_t)s * (Dv + 2) + c];
+      const float4 v = *reinterpret_cast<const float4 *>(p + (int64_t)s * stride + c);
+      const float ws = s_w[s];
+      o.x += ws * v.x; o.y += ws * v.y; o.z += ws * v.z; o.w += ws * v.w;
     }
-    out[nh * Dv + c] = L > 0.f ? o / L : 0.f;
+    *reinterpret_cast<float4 *>(out + nh * Dv + c) = make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
   }
-  if (threadIdx.x == 0) lse[nh] = L > 0.f ? 0.6931471805599453f * (M + log2f(L)) : -INFINITY;
+  if (tid == 0) lse[nh] = L > 0.f ? 0.6931471805599453f * (M + log2f(L)) : -INFINITY;
 }
 
 }  // namespace

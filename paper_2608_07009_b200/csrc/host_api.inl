@@ -159,7 +159,7 @@ struct AttGeom { int splits, tiles_per_split; size_t smem, workspace; };
 int attention_geometry(const hisparse *h, int num_heads, int value_dims, AttGeom *g) {
   const int64_t E = h->d.E;
   if (num_heads < kAttHeads || num_heads % kAttHeads) return HISPARSE_EINVAL;
-  if (E % 32 || !(value_dims == 64 || value_dims == 128 || value_dims == 256 || value_dims == 512) || value_dims > E / 2)
+  if (E % 32 || !(value_dims == 128 || value_dims == 256 || value_dims == 512) || value_dims > E / 2)
     return HISPARSE_EINVAL;
   const int tiles = (h->d.k + kAttTile - 1) / kAttTile;
   const int64_t groups = (int64_t)h->d.N * (num_heads / kAttHeads);
@@ -168,9 +168,9 @@ int attention_geometry(const hisparse *h, int num_heads, int value_dims, AttGeom
   g->tiles_per_split = (tiles + want - 1) / want;
   g->splits = (tiles + g->tiles_per_split - 1) / g->tiles_per_split;
   const size_t row = (size_t)E + kAttPad;
-  g->smem = kAttHeads * row + 2 * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttWarps * 16 * 4 + 16 +
-            (size_t)g->tiles_per_split * kAttTile * 4;
-  g->workspace = (size_t)h->d.N * num_heads * g->splits * (value_dims + 2) * sizeof(float);
+  g->smem = kAttHeads * row + 2 * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttGroups * 16 * 4 +
+            kAttWarps * 32 * 16 + 16 + (size_t)g->tiles_per_split * kAttTile * 4;
+  g->workspace = (size_t)h->d.N * num_heads * g->splits * (value_dims + 4) * sizeof(float);
   return HISPARSE_OK;
 }
 
@@ -581,10 +581,9 @@ int hisparse_sparse_attention(hisparse_t *h, int layer, const void *q_dev, int n
   const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(q_dev);
   float *partial = static_cast<float *>(workspace_dev);
   switch (value_dims) {
-    case 64: rc = launch_attention<2>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
-    case 128: rc = launch_attention<4>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
-    case 256: rc = launch_attention<8>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
-    default: rc = launch_attention<16>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+    case 128: rc = launch_attention<2>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+    case 256: rc = launch_attention<4>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
+    default: rc = launch_attention<8>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
   }
   if (rc) return rc;
   sparse_attention_combine_kernel<<<(unsigned)(h->d.N * num_heads), 128, 0, st>>>(partial, g.splits, value_dims, out_dev, lse_dev);

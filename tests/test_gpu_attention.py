@@ -34,7 +34,7 @@ def check(out, lse, out_ref, lse_ref, vmax):
 @pytest.mark.parametrize("N,H,D,DV,k,B,steps", [
     (3, 16, 576, 512, 256, 512, 3),       # the DSA record: 512-number latent + 64-number rotary key
     (2, 32, 576, 512, 70, 128, 2),        # two head groups, a ragged last tile
-    (5, 16, 128, 64, 33, 64, 2),          # small records, one entry past a tile
+    (5, 16, 144, 128, 33, 64, 2),         # small records (an odd number of k-steps), one entry past a tile
     (1, 16, 256, 256, 512, 1024, 2),      # value = the whole record; many splits for one request
 ])
 def test_attention_over_resolved_tables_matches_the_oracle(N, H, D, DV, k, B, steps):
@@ -117,7 +117,7 @@ def test_attention_edge_rows_and_placement():
         out2, lse2 = gpu.sparse_attention(0, q_d, torch.from_numpy(np.ascontiguousarray(tab_h[:, perm])).to(DEV), DV, 1.0)
         assert torch.allclose(out, out2, atol=2e-2 * float(np.abs(rec0).max())) and torch.allclose(lse[0], lse2[0], atol=4e-3)
         # shapes the kernel does not take are refused before anything is enqueued
-        for heads, dv in ((8, 128), (16, 100), (16, 256)):
+        for heads, dv in ((8, 128), (16, 64), (16, 100), (16, 256)):
             with pytest.raises(HiSparseError) as e:
                 gpu.attention_workspace_bytes(heads, dv)
             assert e.value.code == hs.EINVAL
