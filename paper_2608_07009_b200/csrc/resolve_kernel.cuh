@@ -1070,33 +1070,16 @@ __device__ __forceinline__ int32_t atom_add_s32(uint32_t a, int32_t v) {
   return o;
 }
 
-// What miss_path_cold hands back to a looping block, packed into one word (no locals whose address is taken).
-constexpr uint32_t kColdFetchParity = 1u, kColdOrderParity = 2u, kColdGaveUp = 4u;
-
+// Returns -1 when the block has nothing left to do; otherwise the number of requests it has finished, with `r` the
+// request in which something missed: that request's row and slice are still staged (its barrier's phase is over), its
+// marks are written and its counters cleared, and the caller's general loop takes it from the lookups on.  (Calling the
+// out-of-line miss path from inside this loop made the compiler keep the loop's state in local memory around the call
+// site: ~17 spill instructions per warp and request on a path that never made the call; as a function of its own,
+// out of line, the loop spilled even more.)
 template <int T>
-__device__ __noinline__ uint32_t lean_miss(const DevState &d, const int layer, const int g, const int32_t *sel, int32_t *table,
-                                           int32_t *hits_out, int32_t *misses_out, const int r, const int it, const int tag,
-                                           const bool has_next, const uint32_t t, const uint32_t st, const uint32_t state) {
-  const int k = d.k;
-  const int64_t cap = d.uni_cap;
-  ReqCtx c;
-  c.r = r; c.it = it; c.S = 1; c.layer = layer; c.g = g; c.rg = (int64_t)r * d.G + g;
-  c.cap_r = cap; c.init_len_r = d.uni_init_len; c.p2s_off_r = (int64_t)r * d.G * p2s_stride(cap);
-  c.row = sel + (int64_t)r * k;
-  c.trow = table + (int64_t)r * k;
-  c.arow = d.lpg > 1 ? d.anchor_out + c.rg * k : nullptr;
-  c.hits_out = hits_out; c.misses_out = misses_out;
-  c.has_next = has_next; c.tag = tag;
-  uint32_t fetch_parity = state & kColdFetchParity, order_parity = (state & kColdOrderParity) ? 1u : 0u;
-  bool gave_up = false;
-  miss_path_cold<T, 4>(d, c, t, d.order_t[c.rg], st, fetch_parity, order_parity, gave_up);
-  return fetch_parity | (order_parity ? kColdOrderParity : 0u) | (gave_up ? kColdGaveUp : 0u);
-}
-
-template <int T>
-__device__ __forceinline__ void lean_loop(const DevState &d, const int layer, const int g, const int32_t *__restrict__ sel,
-                                          int32_t *__restrict__ table, int32_t *__restrict__ hits_out,
-                                          int32_t *__restrict__ misses_out, int r, const int stride) {
+__device__ __forceinline__ int lean_loop(const DevState &d, const int g, const int32_t *__restrict__ sel,
+                                         int32_t *__restrict__ table, int32_t *__restrict__ hits_out,
+                                         int32_t *__restrict__ misses_out, int &r, const int stride) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, lane = tid & 31;
   const int k = d.k, B = d.B, N = d.N;
@@ -1105,16 +1088,13 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
   const uint32_t a_marks = a_base + (uint32_t)d.sm_marks;
   const uint32_t a_spare = a_marks + (uint32_t)d.marks_spare;                // a byte that no slot owns
   const uint32_t a_misc = a_base + (uint32_t)d.sm_misc + 128u;              // two sets of 8 ints
-  const uint32_t a_stash = a_base + (uint32_t)d.sm_plan_slot + (uint32_t)tid * 16u;
   const uint32_t stage_bar = a_base + (uint32_t)d.meta_smem + (uint32_t)T * 8u;
   const uint32_t a_row = a_base + (uint32_t)tid * 16u;                      // this thread's four row entries
   const int cap = (int)d.uni_cap, il = (int)d.uni_init_len;
   const bool mine = tid * 4 < k;
   const bool stamp_hits = d.policy != HISPARSE_POLICY_FIFO;
   const int G = d.G;
-  uint32_t state = 0;   // kCold* bits: phases of the fetch / list barriers as the out-of-line path left them
-  int tag = 0;
-  uint32_t parity = 0;
+  int tag = 0, it = 0;
   // a request's resolve count is loaded one request ahead (with the next request's inputs), so that the trip to
   // memory is over when the count is needed
   uint32_t t_ahead = r < N ? d.t[r * G + g] : 0u;
@@ -1123,8 +1103,9 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
   int len = il + na, newest = na > 0 ? il + na - 1 : -2;  // -2: no newest record (a discarded entry is -1)
   if (len > cap) { len = cap; newest = -2; }
   bool more = r < N;
-  for (; more; parity ^= 1u) {
+  for (; more; ++it) {
     const int rg = r * G + g;                       // N * G fits 32 bits (the metadata arrays are indexed by it)
+    const uint32_t parity = (uint32_t)it & 1u;
     const uint32_t a_set = a_misc + parity * 32u;
     if (tag == 255) {
       // the tags start over: forget the old marks (every thread is done with the previous request's)
@@ -1188,18 +1169,10 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
     const bool has_next = rn < N;
     if (has_next) t_ahead = d.t[rn * G + g];
     if (any_miss) {
-      // something missed: the general path, out of line; the thread's missing positions travel through shared memory
-      if (mine) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) sts_s32(a_stash + 4u * i, (pos[i] >= 0 && pos[i] != newest && got[i] < 0) ? pos[i] : -1);
-      }
-      state = lean_miss<T>(d, layer, g, sel, table, hits_out, misses_out, r, (int)parity, tag, has_next, t, st, state);
-      // after a fetch, the next request's inputs can only start once every thread is done with the ring
-      if (__syncthreads_or((state & kColdGaveUp) != 0)) break;
-      if (has_next && tid < 32) lean_stage_issue<T>(d, sel, g, rn, a_base, a_ring, stage_bar);
-      more = has_next;
-      r = rn;
-      continue;
+      // something missed: the general loop takes this request again from its lookups on (the staged row and slice are
+      // untouched, the marks carry this request's tag either way); what this pass counted is forgotten
+      if (tid == 0) { sts_s32(a_set, 0); sts_s32(a_set + 4u, 0); sts_s32(a_set + 8u, 0); sts_s32(a_set + 12u, 0); }
+      return it;
     }
     if (has_next && !gave_up) {
       // the row and the ring are free (every thread consumed its entries before the vote): the next request's inputs
@@ -1246,6 +1219,7 @@ __device__ __forceinline__ void lean_loop(const DevState &d, const int layer, co
     more = has_next;
     r = rn;
   }
+  return -1;
 }
 
 // MINB = thread blocks of this size that must fit one SM (bounds the registers per thread).
@@ -1304,14 +1278,15 @@ resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_
   uint32_t fetch_parity = 0, order_parity = 0;  // phases of this thread's fetch barrier / of the list's staging barrier
   bool gave_up = false;                          // a bounded wait expired: the block takes no further request
 
+  int it = 0;
   if constexpr (LOOP) {
     if (S == 1 && lean_shape(d, sel, table, T)) {
-      lean_loop<T>(d, layer, g, sel, table, hits_out, misses_out, r, stride);
-      return;
+      it = lean_loop<T>(d, g, sel, table, hits_out, misses_out, r, stride);
+      if (it < 0) return;
     }
   }
   // (the wide block never loops: one pass, so that nothing has to stay in registers across requests)
-  for (int it = 0; r < d.N && !gave_up && (LOOP || it == 0); r += stride, ++it) {
+  for (; r < d.N && !gave_up && (LOOP || it == 0); r += stride, ++it) {
     ReqCtx c;
     c.r = r; c.it = it; c.S = S; c.layer = layer; c.g = g;
     c.rg = (int64_t)r * d.G + g;

@@ -289,6 +289,43 @@ def test_narrow_blocks_shapes_groups_and_policies(policy):
     run_trace(w, w.steps, use_prefetch=True, ctas_per_request=2, flags=NARROW, policy=policy, policy_seed=3)
 
 
+@pytest.mark.parametrize("init_len,policy", [(250, hs.POLICY_LRU), (250, hs.POLICY_FIFO), (1500, hs.POLICY_LRU)])
+def test_resident_wave_of_looping_blocks(init_len, policy):
+    """More requests than blocks fit the GPU at once: the launch is one resident wave whose blocks take the requests
+    b, b + blocks, b + 2 blocks, .. one after the other, with the later requests' rows and page-table slices staged
+    ahead (in two buffers when the slice is small enough: init_len 250; in one: init_len 1500).  Requests in which
+    nothing misses and requests with misses alternate at random, so that a block meets every order of the two."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    N, k, B = 6 * sms + 37, 64, 128                 # at most 3 blocks per SM are resident: every block loops
+    rng = np.random.default_rng(init_len + policy)
+    w = tiny_workload(N, 1, 1, k, B, 32, [init_len] * N, steps=8)
+    pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=11)
+    try:
+        assert pair.gpu.launch_geometry()["threads"] == 512
+        for step in range(7):
+            if step % 2 == 1:
+                pair.append()
+            rows = []
+            for r in range(N):
+                res = pair.oracle.slot_pos(r, 0)
+                res = res[res >= 0]
+                if step > 0 and rng.random() < 0.5 and len(res) >= k // 2:     # nothing misses
+                    n = int(rng.integers(k // 2, min(k, len(res)) + 1))
+                    row = rng.choice(res, size=n, replace=False).astype(np.int32)
+                    if pair.oracle.newest(r) >= 0 and n < k and rng.random() < 0.5:
+                        row = np.append(row, np.int32(pair.oracle.newest(r)))
+                    row = rng.permutation(np.concatenate([row, np.full(k - len(row), -1, dtype=np.int32)]))
+                else:
+                    row = inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0]
+                rows.append(row)
+            _, _, m = pair.resolve_and_compare(0, np.stack(rows))
+            assert 0 < int((m == 0).sum()) < N or step == 0
+            pair.compare_state(0)
+        pair.finish()
+    finally:
+        pair.close()
+
+
 def test_block_size_is_chosen_by_the_grid_and_refused_when_it_cannot_fit():
     w = tiny_workload(2, 1, 1, 4, 8, 32, [20, 30])
     pair = Pair(w)
