@@ -1186,16 +1186,43 @@ __device__ __forceinline__ int lean_loop(const DevState &d, const int g, const i
       const uint32_t hit_stamp = 2u * t + 1u;
       const uint32_t a_m = a_marks + (uint32_t)tid;
       int cnt = 0;
-      for (int s0 = 0; s0 < B; s0 += 4 * T) {   // the marks are padded to whole rounds of this loop (padding = 0)
-        uint32_t m[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) m[j] = lds_u8(a_m + (uint32_t)(s0 + j * T));
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const bool hit = m[j] == (uint32_t)tag;
-          if (hit && stamp_hits) lu[s0 + j * T] = hit_stamp;
-          cnt += hit;
+      if (stamp_hits) {
+        // four slots per round, written out in PTX: four loads, four compares, four predicated stores, the count
+        // (the marks are padded to whole rounds of this loop, padding = 0)
+        for (int s0 = 0; s0 < B; s0 += 4 * T) {
+          uint32_t c4;
+          asm volatile(
+              "{\n"
+              ".reg .pred p0, p1, p2, p3;\n"
+              ".reg .u32 m0, m1, m2, m3, c0, c1, c2, c3;\n"
+              "ld.shared.u8 m0, [%1];\n"
+              "ld.shared.u8 m1, [%1+%5];\n"
+              "ld.shared.u8 m2, [%1+%6];\n"
+              "ld.shared.u8 m3, [%1+%7];\n"
+              "setp.eq.u32 p0, m0, %2;\n"
+              "setp.eq.u32 p1, m1, %2;\n"
+              "setp.eq.u32 p2, m2, %2;\n"
+              "setp.eq.u32 p3, m3, %2;\n"
+              "@p0 st.global.u32 [%3], %4;\n"
+              "@p1 st.global.u32 [%3+%8], %4;\n"
+              "@p2 st.global.u32 [%3+%9], %4;\n"
+              "@p3 st.global.u32 [%3+%10], %4;\n"
+              "selp.u32 c0, 1, 0, p0;\n"
+              "selp.u32 c1, 1, 0, p1;\n"
+              "selp.u32 c2, 1, 0, p2;\n"
+              "selp.u32 c3, 1, 0, p3;\n"
+              "add.u32 c0, c0, c1;\n"
+              "add.u32 c2, c2, c3;\n"
+              "add.u32 %0, c0, c2;\n"
+              "}"
+              : "=r"(c4)
+              : "r"(a_m + (uint32_t)s0), "r"((uint32_t)tag), "l"(lu + s0), "r"(hit_stamp), "n"(T), "n"(2 * T), "n"(3 * T),
+                "n"(4 * T), "n"(8 * T), "n"(12 * T)
+              : "memory");
+          cnt += (int)c4;
         }
+      } else {   // FIFO: a hit changes no stamp; only the distinct slots are counted
+        for (int s0 = 0; s0 < B; s0 += T) cnt += lds_u8(a_m + (uint32_t)s0) == (uint32_t)tag;
       }
       cnt = __reduce_add_sync(0xffffffffu, cnt);
       if (lane == 0 && cnt) red_add_s32(a_set + 12u, cnt);
