@@ -28,6 +28,8 @@ constexpr int kAttGroups = kAttTile / 8;   // groups of 8 records (one n-tile of
 constexpr int kAttThreads = kAttWarps * 32;
 constexpr int kAttHeads = 16;       // heads per block (one m16 row block)
 constexpr int kAttPad = 16;         // bytes of padding per staged row
+constexpr int kAttStages = 2;       // tiles in the gather ring
+constexpr int kAttMaxQuerySteps = 9;   // k-steps of the query per warp at most: records of up to 4 x 9 x 16 = 576 numbers
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -50,8 +52,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Partial result of one (request, head, split): Dv unnormalised output numbers, then the running maximum (base 2) and
 // the sum of the weights, padded to Dv + 4 floats so that rows stay 16-byte aligned.
-// NV = Dv / 64 = 8-wide output tiles per warp (Dv = 512 -> 8).
-template <int NV>
+// NV = Dv / 64 = 8-wide output tiles per warp (Dv = 512 -> 8).  KQ = k-steps (of 16 numbers) of the query that a warp
+// keeps in registers = ceil(D / 64) at most (D = 576 -> 9).
+template <int NV, int KQ>
 __global__ void __launch_bounds__(kAttThreads, 2)
 sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const int32_t *__restrict__ table, const int k,
                         const __nv_bfloat16 *__restrict__ q, const int H, const float scale_log2e, const int splits,
@@ -69,14 +72,14 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
 
   unsigned char *s_q = smem_raw;                                         // [16][row_bytes]
   unsigned char *s_kv = s_q + kAttHeads * row_bytes;                     // [2][kAttTile][row_bytes]
-  unsigned char *s_p = s_kv + 2 * kAttTile * row_bytes;                  // [16][kAttTile * 2 + 16] bf16 weights
+  unsigned char *s_p = s_kv + kAttStages * kAttTile * row_bytes;         // [16][kAttTile * 2 + 16] bf16 weights
   float *s_red = reinterpret_cast<float *>(s_p + kAttHeads * (kAttTile * 2 + kAttPad));   // [kAttGroups][16]
-  float4 *s_part = reinterpret_cast<float4 *>(s_red + kAttGroups * 16);                    // [kAttWarps][32]: half scores
-  unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_part + kAttWarps * 32);   // [2]
-  int32_t *s_tab = reinterpret_cast<int32_t *>(s_bar + 2);               // [per]: this split's table entries
+  float4 *s_part = reinterpret_cast<float4 *>(s_red + kAttGroups * 16);                    // [kAttWarps][2][32]: partial scores
+  unsigned long long *s_bar = reinterpret_cast<unsigned long long *>(s_part + kAttWarps * 64);   // [kAttStages]
+  int32_t *s_tab = reinterpret_cast<int32_t *>(s_bar + (kAttStages + 1) / 2 * 2);   // [per]: this split's table entries
   constexpr int p_stride = kAttTile * 2 + kAttPad;
 
-  if (tid < 2) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(s_bar + tid)), "r"(kAttTile) : "memory");
+  if (tid < kAttStages) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(s_bar + tid)), "r"(kAttTile) : "memory");
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   // this split's slice of the row (-1 past its end): read once, so that neither the gather nor the masking waits
   // for global memory inside the tile loop
@@ -99,8 +102,8 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   auto gather = [&](const int t) {
     if (tid >= kAttTile || t >= ntiles) return;
     const int32_t rec = s_tab[t * kAttTile + tid];
-    unsigned char *dst = s_kv + ((t & 1) * kAttTile + tid) * row_bytes;
-    const uint32_t bar = smem_u32(s_bar + (t & 1));
+    unsigned char *dst = s_kv + ((t % kAttStages) * kAttTile + tid) * row_bytes;
+    const uint32_t bar = smem_u32(s_bar + (t % kAttStages));
     if (rec >= 0) {
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)E) : "memory");
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -111,13 +114,28 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
     }
   };
-  gather(0);
-  gather(1);
+#pragma unroll
+  for (int i = 0; i < kAttStages; ++i) gather(i);
 
   const int r0 = lane >> 2;                 // this thread's accumulator rows are r0 and r0 + 8
-  const int grp = warp & (kAttGroups - 1);  // the 8 records of a tile this warp scores ...
-  const bool half = warp >= kAttGroups;     // ... over the lower or the upper half of D
-  const int d_mid = ((D / 16 + 1) / 2) * 16, d_lo = half ? d_mid : 0, d_hi = half ? D : d_mid;
+  // Scores: warp w multiplies the records 16 (w & 1) .. + 15 of a tile (two n-tiles) with the query over the k-steps
+  // [ks_lo, ks_hi) = quarter w >> 1 of D; its slice of the query never changes, so it lives in registers as A
+  // fragments (read from shared memory every tile, the query made up half of the kernel's shared-memory traffic).
+  const int rh = warp & 1, dq = warp >> 1;
+  const int KS = D / 16, ks_lo = KS * dq / 4, ks_hi = KS * (dq + 1) / 4;
+  uint32_t qa[KQ][4];
+  {
+    const uint32_t a_addr = smem_u32(s_q) + (uint32_t)((lane & 15) * row_bytes + (lane >> 4) * 16);
+#pragma unroll
+    for (int i = 0; i < KQ; ++i) {
+      if (ks_lo + i < ks_hi) ldsm_x4(qa[i], a_addr + (uint32_t)(ks_lo + i) * 32u);
+      else qa[i][0] = qa[i][1] = qa[i][2] = qa[i][3] = 0u;
+    }
+  }
+  // Softmax: warp w owns n-tile w & 3 of the summed scores (the warps w and w + 4 hold the same numbers; the lower
+  // four write the weights)
+  const int grp = warp & (kAttGroups - 1);
+  const bool half = warp >= kAttGroups;
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   float acc[NV][4];
 #pragma unroll
@@ -125,46 +143,40 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   bool timed_out = false;
 
   for (int t = 0; t < ntiles; ++t) {
-    if (!mbar_wait_bounded(smem_u32(s_bar + (t & 1)), (uint32_t)((t >> 1) & 1))) timed_out = true;
-    const unsigned char *kv = s_kv + (t & 1) * kAttTile * row_bytes;
-    // S = Q K^T for this warp's 8 records over its half of D: 16 x 8, k-steps of 16
-    // (four independent accumulators, summed at the end: one accumulator would make the MMAs one dependent chain)
+    if (!mbar_wait_bounded(smem_u32(s_bar + (t % kAttStages)), (uint32_t)((t / kAttStages) & 1))) timed_out = true;
+    const unsigned char *kv = s_kv + (t % kAttStages) * kAttTile * row_bytes;
+    // S = Q K^T for this warp's 16 records over its quarter of D: two 16 x 8 n-tiles, k-steps of 16, two accumulators
+    // per n-tile (one would make the MMAs one dependent chain).  One ldmatrix.x4 per k-step: records 0-7 / 8-15 of the
+    // warp's half, lower / upper 8 numbers of the k-step.
     float sc[4];
     {
-      float part[4][4];
+      float part[2][2][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) part[i][0] = part[i][1] = part[i][2] = part[i][3] = 0.f;
-      const uint32_t a_addr = smem_u32(s_q) + (uint32_t)((lane & 15) * row_bytes + (lane >> 4) * 16);
-      const uint32_t b_addr = smem_u32(kv) + (uint32_t)((grp * 8 + (lane & 7)) * row_bytes + (lane >> 3) * 16);
-      int d0 = d_lo;
-#pragma unroll 2
-      for (; d0 + 64 <= d_hi; d0 += 64) {        // four k-steps per iteration (two ldmatrix.x4 of B)
-        uint32_t a[4][4], b0[4], b1[4];
-        ldsm_x4(b0, b_addr + (uint32_t)d0 * 2u);
-        ldsm_x4(b1, b_addr + (uint32_t)(d0 + 32) * 2u);
+      for (int i = 0; i < 2; ++i)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) ldsm_x4(a[i], a_addr + (uint32_t)(d0 + 16 * i) * 2u);
-        mma_bf16(part[0], a[0], b0[0], b0[1]);
-        mma_bf16(part[1], a[1], b0[2], b0[3]);
-        mma_bf16(part[2], a[2], b1[0], b1[1]);
-        mma_bf16(part[3], a[3], b1[2], b1[3]);
+        for (int j = 0; j < 2; ++j) part[i][j][0] = part[i][j][1] = part[i][j][2] = part[i][j][3] = 0.f;
+      const uint32_t b_addr = smem_u32(kv) + (uint32_t)((rh * 16 + (lane & 7) + (lane >> 4) * 8) * row_bytes + ((lane >> 3) & 1) * 16) +
+                              (uint32_t)ks_lo * 32u;
+#pragma unroll
+      for (int i = 0; i < KQ; ++i) {
+        if (ks_lo + i < ks_hi) {   // (uniform in the warp)
+          uint32_t b[4];
+          ldsm_x4(b, b_addr + (uint32_t)i * 32u);
+          mma_bf16(part[0][i & 1], qa[i], b[0], b[1]);
+          mma_bf16(part[1][i & 1], qa[i], b[2], b[3]);
+        }
       }
-      for (; d0 < d_hi; d0 += 16) {              // what is left of the half (a multiple of 16)
-        uint32_t a[4], b[4];
-        ldsm_x4(b, b_addr + (uint32_t)d0 * 2u);   // its upper half may lie past the row's end: not used
-        ldsm_x4(a, a_addr + (uint32_t)d0 * 2u);
-        mma_bf16(part[0], a, b[0], b[1]);
-      }
-      const float4 mine = make_float4((part[0][0] + part[1][0]) + (part[2][0] + part[3][0]),
-                                      (part[0][1] + part[1][1]) + (part[2][1] + part[3][1]),
-                                      (part[0][2] + part[1][2]) + (part[2][2] + part[3][2]),
-                                      (part[0][3] + part[1][3]) + (part[2][3] + part[3][3]));
-      s_part[warp * 32 + lane] = mine;
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+        s_part[(warp * 2 + nt) * 32 + lane] = make_float4(part[nt][0][0] + part[nt][1][0], part[nt][0][1] + part[nt][1][1],
+                                                         part[nt][0][2] + part[nt][1][2], part[nt][0][3] + part[nt][1][3]);
       __syncthreads();
-      const float4 other = s_part[(warp ^ kAttGroups) * 32 + lane];   // the same records, the other half of D
-      // (added in a fixed order, so that both warps of a pair hold bit-identical scores)
-      const float4 lo4 = half ? other : mine, hi4 = half ? mine : other;
-      sc[0] = lo4.x + hi4.x; sc[1] = lo4.y + hi4.y; sc[2] = lo4.z + hi4.z; sc[3] = lo4.w + hi4.w;
+      // n-tile grp = records 8 grp .. + 7 was scored by the warps (grp >> 1) + 2 dq as their n-tile grp & 1: the four
+      // quarters of D, added in a fixed order (so that both warps that own the n-tile hold bit-identical scores)
+      const int src = grp * 32 + lane;
+      const float4 p0 = s_part[src], p1 = s_part[src + 4 * 32], p2 = s_part[src + 8 * 32], p3 = s_part[src + 12 * 32];
+      sc[0] = (p0.x + p1.x) + (p2.x + p3.x); sc[1] = (p0.y + p1.y) + (p2.y + p3.y);
+      sc[2] = (p0.z + p1.z) + (p2.z + p3.z); sc[3] = (p0.w + p1.w) + (p2.w + p3.w);
     }
     // mask padding, scale into the base-2 domain, row maxima over the tile
     const int jbase = t * kAttTile + grp * 8 + 2 * (lane & 3);
@@ -226,7 +238,7 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
       }
     }
     __syncthreads();   // every warp is done with this tile's buffer, the weights and the maxima
-    gather(t + 2);
+    gather(t + kAttStages);
   }
 
   // partial sums of the weights: across the quad, then across the record groups (one warp of each pair reports)

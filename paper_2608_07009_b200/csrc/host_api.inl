@@ -159,7 +159,8 @@ struct AttGeom { int splits, tiles_per_split; size_t smem, workspace; };
 int attention_geometry(const hisparse *h, int num_heads, int value_dims, AttGeom *g) {
   const int64_t E = h->d.E;
   if (num_heads < kAttHeads || num_heads % kAttHeads) return HISPARSE_EINVAL;
-  if (E % 32 || !(value_dims == 128 || value_dims == 256 || value_dims == 512) || value_dims > E / 2)
+  if (E % 32 || E > 2 * 64 * kAttMaxQuerySteps || !(value_dims == 128 || value_dims == 256 || value_dims == 512) ||
+      value_dims > E / 2)
     return HISPARSE_EINVAL;
   const int tiles = (h->d.k + kAttTile - 1) / kAttTile;
   const int64_t groups = (int64_t)h->d.N * (num_heads / kAttHeads);
@@ -168,24 +169,35 @@ int attention_geometry(const hisparse *h, int num_heads, int value_dims, AttGeom
   g->tiles_per_split = (tiles + want - 1) / want;
   g->splits = (tiles + g->tiles_per_split - 1) / g->tiles_per_split;
   const size_t row = (size_t)E + kAttPad;
-  g->smem = kAttHeads * row + 2 * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttGroups * 16 * 4 +
-            kAttWarps * 32 * 16 + 16 + (size_t)g->tiles_per_split * kAttTile * 4;
+  g->smem = kAttHeads * row + kAttStages * kAttTile * row + kAttHeads * (kAttTile * 2 + kAttPad) + kAttGroups * 16 * 4 +
+            kAttWarps * 64 * 16 + (kAttStages + 1) / 2 * 16 + (size_t)g->tiles_per_split * kAttTile * 4;
   g->workspace = (size_t)h->d.N * num_heads * g->splits * (value_dims + 4) * sizeof(float);
   return HISPARSE_OK;
 }
 
-template <int NV>
-int launch_attention(hisparse *h, const AttGeom &g, const uint8_t *pool, const int32_t *table, const __nv_bfloat16 *q,
-                     int num_heads, float scale, float *partial, cudaStream_t st) {
+template <int NV, int KQ>
+int launch_attention_kq(hisparse *h, const AttGeom &g, const uint8_t *pool, const int32_t *table, const __nv_bfloat16 *q,
+                        int num_heads, float scale, float *partial, cudaStream_t st) {
   int optin = 0;
   HS_CUDA(cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
   if (g.smem > (size_t)optin) return HISPARSE_EINVAL;
-  HS_CUDA(cudaFuncSetAttribute(sparse_attention_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem));
+  HS_CUDA(cudaFuncSetAttribute(sparse_attention_kernel<NV, KQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem));
   const dim3 grid((unsigned)(h->d.N * g.splits), (unsigned)(num_heads / kAttHeads));
-  sparse_attention_kernel<NV><<<grid, kAttThreads, g.smem, st>>>(pool, h->d.E, table, h->d.k, q, num_heads,
-                                                                 scale * 1.4426950408889634f, g.splits, partial, h->d.status);
+  sparse_attention_kernel<NV, KQ><<<grid, kAttThreads, g.smem, st>>>(pool, h->d.E, table, h->d.k, q, num_heads,
+                                                                     scale * 1.4426950408889634f, g.splits, partial, h->d.status);
   HS_CUDA(cudaGetLastError());
   return HISPARSE_OK;
+}
+
+// The kernel keeps a quarter of the query's k-steps (16 numbers each) per warp in registers: the instantiation with the
+// smallest array that holds them.
+template <int NV>
+int launch_attention(hisparse *h, const AttGeom &g, const uint8_t *pool, const int32_t *table, const __nv_bfloat16 *q,
+                     int num_heads, float scale, float *partial, cudaStream_t st) {
+  const int steps = (int)(h->d.E / 32), per_warp = (steps + 3) / 4;
+  if (per_warp <= 3) return launch_attention_kq<NV, 3>(h, g, pool, table, q, num_heads, scale, partial, st);
+  if (per_warp <= 5) return launch_attention_kq<NV, 5>(h, g, pool, table, q, num_heads, scale, partial, st);
+  return launch_attention_kq<NV, kAttMaxQuerySteps>(h, g, pool, table, q, num_heads, scale, partial, st);
 }
 
 }  // namespace
