@@ -95,14 +95,20 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   }
   __syncthreads();
 
-  // Gather of tile t into buffer t & 1: thread j < kAttTile brings record j.  A valid entry is one bulk copy; padding
-  // (or an entry past the split's end) is zero-filled by plain stores, so that 0 weight times the row is 0, not NaN.
+  // Gather of tile t into buffer t % kAttStages: the first four lanes of every warp bring one record each.  A valid
+  // entry is one bulk copy; padding (or an entry past the split's end) is zero-filled by plain stores, so that 0 weight
+  // times the row is 0, not NaN.  Four per warp rather than 32 lanes of one warp: a warp issues the bulk copies of its
+  // lanes one after the other (the instruction takes its operands from uniform registers), ~65 cycles each, so one
+  // warp spent ~2100 cycles per tile issuing, as long as the tile's whole arithmetic, with the other warps waiting for
+  // it at the next barrier.
   // (16-byte cp.async copies by all threads instead: 32.7 us against 30 us; asking the later tiles' records into L2
   // with one prefetch each at the start: 37 us.  Both measured on the C2 shape, neither kept.)
+  constexpr int kPerWarp = kAttTile / kAttWarps;   // records each warp brings
   auto gather = [&](const int t) {
-    if (tid >= kAttTile || t >= ntiles) return;
-    const int32_t rec = s_tab[t * kAttTile + tid];
-    unsigned char *dst = s_kv + ((t % kAttStages) * kAttTile + tid) * row_bytes;
+    if (lane >= kPerWarp || t >= ntiles) return;
+    const int j = warp * kPerWarp + lane;
+    const int32_t rec = s_tab[t * kAttTile + j];
+    unsigned char *dst = s_kv + ((t % kAttStages) * kAttTile + j) * row_bytes;
     const uint32_t bar = smem_u32(s_bar + (t % kAttStages));
     if (rec >= 0) {
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)E) : "memory");
