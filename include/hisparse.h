@@ -194,7 +194,7 @@ const void *hisparse_layer_pool(const hisparse_t *h, int layer);
  * valid entry gives out = 0, lse = -inf.
  *   q_dev      bf16  [N][num_heads][D], 16-byte aligned; num_heads a multiple of 16
  *   out_dev    float [N][num_heads][value_dims]; lse_dev float [N][num_heads]
- *   value_dims 128, 256 or 512, at most D; E a multiple of 32
+ *   value_dims 128, 256 or 512, at most D; E a multiple of 32, at most 1152 (records of up to 576 numbers)
  *   workspace_dev  device scratch of at least hisparse_attention_workspace_bytes bytes (the partial results of the
  *                  blocks that share one row), caller-owned so that the call allocates nothing; 16-byte aligned
  * Arithmetic: bf16 products accumulated in fp32 on the tensor cores, softmax weights rounded to bf16 before they

@@ -13,12 +13,14 @@
 // blocks per SM, and a second small kernel combines the splits.
 //
 // Block = 8 warps, one request, one group of 16 heads, one contiguous split of the row's k entries, tiles of 32
-// records.  Per tile: S = Q K^T (warp w: records 8 (w & 3) .. + 7 over one half of D, the two halves added through
-// shared memory), running row maximum across the record groups through shared memory, P = exp(S - m) rounded to
-// bf16 into shared memory, O = alpha O + P V (warp w: value dims [Dv/8 w, Dv/8 (w+1)), fp32 accumulators in
-// registers).  Eight warps rather than four: a tile is a serial chain of ldmatrix -> mma -> maximum -> exp -> mma with
-// block barriers in between, and with 8 warps per SM the schedulers issued on 17 % of their cycles.  Rows of the tile are padded by 16 bytes in shared memory,
-// which makes every ldmatrix phase hit 8 different bank groups (a 1152-byte stride would put all rows on one).
+// records.  Per tile: S = Q K^T (warp w: records 16 (w & 1) .. + 15 over quarter w >> 1 of D, with its slice of the
+// query held in registers as A fragments and ONE ldmatrix.x4 of records per k-step; the four quarters are added through
+// shared memory), running row maximum across the record groups through shared memory, P = exp(S - m) rounded to bf16
+// into shared memory, O = alpha O + P V (warp w: value dims [Dv/8 w, Dv/8 (w+1)), fp32 accumulators in registers).
+// Eight warps rather than four: a tile is a serial chain of ldmatrix -> mma -> maximum -> exp -> mma with block
+// barriers in between.  Rows of the tile are padded by 16 bytes in shared memory, which makes every ldmatrix phase
+// hit 8 different bank groups (a 1152-byte stride would put all rows on one).  The combine kernel is launched with
+// programmatic dependent launch, so that its launch latency hides under this kernel's tail.
 
 namespace {
 
@@ -102,7 +104,9 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
   // warp spent ~2100 cycles per tile issuing, as long as the tile's whole arithmetic, with the other warps waiting for
   // it at the next barrier.
   // (16-byte cp.async copies by all threads instead: 32.7 us against 30 us; asking the later tiles' records into L2
-  // with one prefetch each at the start: 37 us.  Both measured on the C2 shape, neither kept.)
+  // with one prefetch each at the start: 37 us; a ninth warp that only gathers: with bulk copies 38 us, with cp.async
+  // 59 us, against 26.5 us; requesting the first tiles before the table slice and the query are loaded: no change.
+  // All measured on the C2 shape, none kept.)
   constexpr int kPerWarp = kAttTile / kAttWarps;   // records each warp brings
   auto gather = [&](const int t) {
     if (lane >= kPerWarp || t >= ntiles) return;
@@ -247,6 +251,7 @@ sparse_attention_kernel(const uint8_t *__restrict__ pool, const int64_t E, const
     gather(t + kAttStages);
   }
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may be scheduled from here on
   // partial sums of the weights: across the quad, then across the record groups (one warp of each pair reports)
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
@@ -288,6 +293,7 @@ sparse_attention_combine_kernel(const float *__restrict__ partial, const int spl
   const int64_t nh = blockIdx.x;
   const int stride = Dv + 4;
   const float *p = partial + nh * splits * stride;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the attention kernel's partial results are complete and visible
   const float m = tid < splits ? p[(int64_t)tid * stride + Dv] : -INFINITY;
   const float l = tid < splits ? p[(int64_t)tid * stride + Dv + 1] : 0.f;
   float M = m;

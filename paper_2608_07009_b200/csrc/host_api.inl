@@ -598,8 +598,21 @@ int hisparse_sparse_attention(hisparse_t *h, int layer, const void *q_dev, int n
     default: rc = launch_attention<8>(h, g, pool, slot_table_dev, q, num_heads, scale, partial, st); break;
   }
   if (rc) return rc;
-  sparse_attention_combine_kernel<<<(unsigned)(h->d.N * num_heads), 128, 0, st>>>(partial, g.splits, value_dims, out_dev, lse_dev);
-  HS_CUDA(cudaGetLastError());
+  {
+    // programmatic dependent launch: the combine kernel is scheduled while the attention kernel drains (it waits for
+    // the partial results with griddepcontrol.wait), which hides its launch latency
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(h->d.N * num_heads));
+    cfg.blockDim = dim3(128);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const float *partial_c = partial;
+    const int splits = g.splits;
+    HS_CUDA(cudaLaunchKernelEx(&cfg, sparse_attention_combine_kernel, partial_c, splits, value_dims, out_dev, lse_dev));
+  }
   return HISPARSE_OK;
 }
 

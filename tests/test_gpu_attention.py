@@ -125,3 +125,13 @@ def test_attention_edge_rows_and_placement():
         gpu.close()
         for h in hist:
             h.free()
+    # records longer than 576 numbers: the kernel's query registers are sized for them, anything longer is refused
+    hist = [HostHistory(1, 40, 1280)]
+    gpu = HiSparse(1, 1, 1, 16, 8, 1280, [40], [40], hist)
+    try:
+        with pytest.raises(HiSparseError) as e:
+            gpu.attention_workspace_bytes(16, 512)
+        assert e.value.code == hs.EINVAL
+    finally:
+        gpu.close()
+        hist[0].free()
