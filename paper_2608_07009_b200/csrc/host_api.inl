@@ -310,9 +310,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   if ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) && (c->flags & HISPARSE_FLAG_WIDE_BLOCKS)) return fail(HISPARSE_EINVAL);
   h->T = kThreads; h->minb = 1;
   if (want_small) {
-    const char *env = getenv("HISPARSE_BLOCKS_PER_SM");   // tuning knob: 2 or 3 narrow blocks per SM
-    const int first = env && atoi(env) == 2 ? 2 : 3;
-    for (int per_sm = first; per_sm >= 2 && h->T == kThreads; --per_sm)
+    for (int per_sm = 3; per_sm >= 2 && h->T == kThreads; --per_sm)   // three narrow blocks per SM if they fit, else two
       if (try_small(per_sm)) { h->T = kThreadsSmall; h->minb = per_sm; }
     if (h->T == kThreads && (c->flags & HISPARSE_FLAG_NARROW_BLOCKS)) return fail(HISPARSE_EINVAL);
   }
@@ -353,8 +351,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   if (h->S == 1 && h->T == kThreadsSmall) {
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, h->T, h->resolve_smem) != cudaSuccess) return fail(HISPARSE_ECUDA);
-    const char *env = getenv("HISPARSE_RESIDENT_WAVE");
-    if (per_sm >= 1 && !(env && atoi(env) == 0)) h->clusters = std::min(N, per_sm * sm_count);
+    if (per_sm >= 1) h->clusters = std::min(N, per_sm * sm_count);
   }
 
 #define HS_TRY(expr) do { int rc_ = (expr); if (rc_) return fail(rc_); } while (0)

@@ -289,12 +289,14 @@ def test_narrow_blocks_shapes_groups_and_policies(policy):
     run_trace(w, w.steps, use_prefetch=True, ctas_per_request=2, flags=NARROW, policy=policy, policy_seed=3)
 
 
-@pytest.mark.parametrize("init_len,policy", [(250, hs.POLICY_LRU), (250, hs.POLICY_FIFO), (1500, hs.POLICY_LRU)])
+@pytest.mark.parametrize("init_len,policy", [(250, hs.POLICY_LRU), (250, hs.POLICY_FIFO), (1500, hs.POLICY_LRU),
+                                             (700, hs.POLICY_RANDOM)])
 def test_resident_wave_of_looping_blocks(init_len, policy):
     """More requests than blocks fit the GPU at once: the launch is one resident wave whose blocks take the requests
-    b, b + blocks, b + 2 blocks, .. one after the other, with the later requests' rows and page-table slices staged
-    ahead (in two buffers when the slice is small enough: init_len 250; in one: init_len 1500).  Requests in which
-    nothing misses and requests with misses alternate at random, so that a block meets every order of the two."""
+    b, b + blocks, b + 2 blocks, .. one after the other, with the next request's row and page-table slice staged
+    ahead.  Requests in which nothing misses and requests with misses alternate at random, so that a block meets
+    every order of the two: it runs the short loop until its first request with a miss and the general loop from
+    there on."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     N, k, B = 6 * sms + 37, 64, 128                 # at most 3 blocks per SM are resident: every block loops
     rng = np.random.default_rng(init_len + policy)
