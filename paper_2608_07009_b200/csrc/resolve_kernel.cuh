@@ -1095,6 +1095,25 @@ __device__ __forceinline__ int lean_loop(const DevState &d, const int g, const i
   const bool stamp_hits = d.policy != HISPARSE_POLICY_FIFO;
   const int G = d.G;
   int tag = 0, it = 0;
+  // The counters of a request are read, reported and cleared by the first thread one request later, behind the block
+  // barrier that follows the staging wait (the two sets of counters alternate): that saves the barrier the counts
+  // would otherwise need right after the stamp pass, one of three per request.
+  int r_prev = -1;
+  uint32_t t_prev = 0, set_prev = 0;
+  auto finish = [&](const int rf, const uint32_t tf, const uint32_t set) {   // first thread only
+    const int rgf = rf * G + g;
+    const int distinct = lds_s32(set + 12u), selected = lds_s32(set + 4u), isnew = lds_s32(set + 8u);
+    if (distinct != selected) atomicOr(d.status, HISPARSE_STATUS_DUPLICATE);  // a resident position was selected twice
+    const int nhits = distinct + (isnew ? 1 : 0);
+    sts_s32(set, 0); sts_s32(set + 4u, 0); sts_s32(set + 8u, 0); sts_s32(set + 12u, 0);  // for the request after the next
+    hits_out[rf] = nhits;
+    misses_out[rf] = 0;
+    d.anchor_hits[rgf] = nhits;
+    d.anchor_misses[rgf] = 0;
+    d.plan_n[rgf] = 0;
+    d.t[rgf] = tf;
+    if (!stamp_hits) d.order_t[rgf] = tf;
+  };
   // a request's resolve count is loaded one request ahead (with the next request's inputs), so that the trip to
   // memory is over when the count is needed
   uint32_t t_ahead = r < N ? d.t[r * G + g] : 0u;
@@ -1108,8 +1127,9 @@ __device__ __forceinline__ int lean_loop(const DevState &d, const int g, const i
     const uint32_t parity = (uint32_t)it & 1u;
     const uint32_t a_set = a_misc + parity * 32u;
     if (tag == 255) {
-      // the tags start over: forget the old marks (every thread is done with the previous request's)
+      // the tags start over: forget the old marks, once every thread is done with the previous request's
       tag = 0;
+      __syncthreads();
       for (int i = tid * 16; i < B; i += T * 16) *reinterpret_cast<uint4 *>(smem_raw + d.sm_marks + i) = make_uint4(0, 0, 0, 0);
       __syncthreads();
     }
@@ -1123,6 +1143,7 @@ __device__ __forceinline__ int lean_loop(const DevState &d, const int g, const i
     uint32_t st = 0;
     bool gave_up = false;
     if (__syncthreads_or(!landed)) { st = HISPARSE_STATUS_TIMEOUT; gave_up = true; }
+    if (tid == 0 && r_prev >= 0) finish(r_prev, t_prev, set_prev);   // (its stamp pass is over)
     int4 x = make_int4(-1, -1, -1, -1);
     if (mine && !gave_up) x = lds_v4(a_row);
     int32_t pos[4] = {x.x, x.y, x.z, x.w};
@@ -1227,24 +1248,17 @@ __device__ __forceinline__ int lean_loop(const DevState &d, const int g, const i
       cnt = __reduce_add_sync(0xffffffffu, cnt);
       if (lane == 0 && cnt) red_add_s32(a_set + 12u, cnt);
     }
-    __syncthreads();  // the counts are complete, and the marks may be written again
-    if (tid == 0) {
-      const int distinct = lds_s32(a_set + 12u), selected = lds_s32(a_set + 4u), isnew = lds_s32(a_set + 8u);
-      if (distinct != selected) st |= HISPARSE_STATUS_DUPLICATE;  // a resident position was selected twice
-      const int nhits = distinct + (isnew ? 1 : 0);
-      sts_s32(a_set, 0); sts_s32(a_set + 4u, 0); sts_s32(a_set + 8u, 0); sts_s32(a_set + 12u, 0);  // for the request after the next
-      hits_out[r] = nhits;
-      misses_out[r] = 0;
-      d.anchor_hits[rg] = nhits;
-      d.anchor_misses[rg] = 0;
-      d.plan_n[rg] = 0;
-      d.t[rg] = t;
-      if (!stamp_hits) d.order_t[rg] = t;
-    }
     if (st) atomicOr(d.status, st);
+    r_prev = r;
+    t_prev = t;
+    set_prev = a_set;
     if (gave_up) break;
     more = has_next;
     r = rn;
+  }
+  if (r_prev >= 0) {   // the block's last request
+    __syncthreads();
+    if (tid == 0) finish(r_prev, t_prev, set_prev);
   }
   return -1;
 }
