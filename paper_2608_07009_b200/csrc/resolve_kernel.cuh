@@ -1135,6 +1135,16 @@ __device__ __forceinline__ int lean_loop(const DevState &d, const int g, const i
     }
     ++tag;
     const uint32_t t = t_ahead + 1u;
+    if (tid >= T - 2 && r + 2 * stride < N) {
+      // the request after the next: its row and slice start their way from HBM to L2 now, two requests ahead of
+      // their use (the staging copy of one request ahead then reads L2)
+      const int r2 = r + 2 * stride;
+      const bool is_row = tid == T - 2;
+      const char *p = is_row ? reinterpret_cast<const char *>(sel + (int64_t)r2 * k)
+                             : reinterpret_cast<const char *>(d.pos2slot + ((int64_t)r2 * G + g) * p2s_stride(cap));
+      const uint32_t n = is_row ? (uint32_t)k * 4u : (uint32_t)p2s_stride(cap) * 2u;
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(n) : "memory");
+    }
     bool landed = true;
     if (tid < 32 && !mbar_wait_bounded(stage_bar, parity)) {
       mbar_wait_bounded(stage_bar, parity);
