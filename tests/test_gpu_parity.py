@@ -289,18 +289,20 @@ def test_narrow_blocks_shapes_groups_and_policies(policy):
     run_trace(w, w.steps, use_prefetch=True, ctas_per_request=2, flags=NARROW, policy=policy, policy_seed=3)
 
 
-@pytest.mark.parametrize("init_len,policy", [(250, hs.POLICY_LRU), (250, hs.POLICY_FIFO), (1500, hs.POLICY_LRU),
-                                             (700, hs.POLICY_RANDOM)])
-def test_resident_wave_of_looping_blocks(init_len, policy):
+@pytest.mark.parametrize("init_len,policy,k,B", [(250, hs.POLICY_LRU, 64, 128), (250, hs.POLICY_FIFO, 64, 128),
+                                                 (1500, hs.POLICY_LRU, 64, 128), (700, hs.POLICY_RANDOM, 64, 128),
+                                                 (3000, hs.POLICY_LRU, 512, 1100), (40000, hs.POLICY_LRU, 100, 300)])
+def test_resident_wave_of_looping_blocks(init_len, policy, k, B):
     """More requests than blocks fit the GPU at once: the launch is one resident wave whose blocks take the requests
     b, b + blocks, b + 2 blocks, .. one after the other, with the next request's row and page-table slice staged
     ahead.  Requests in which nothing misses and requests with misses alternate at random, so that a block meets
     every order of the two: it runs the short loop until its first request with a miss and the general loop from
     there on."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    N, k, B = 6 * sms + 37, 64, 128                 # at most 3 blocks per SM are resident: every block loops
+    N = (6 if k <= 64 else 3) * sms + 37            # at most 3 blocks per SM are resident: every block loops
+    # (init_len 40000: a page-table slice too long to stage, so the blocks never enter the short loop)
     rng = np.random.default_rng(init_len + policy)
-    w = tiny_workload(N, 1, 1, k, B, 32, [init_len] * N, steps=8)
+    w = tiny_workload(N, 1, 1, k, B, 16 if init_len > 10000 else 32, [init_len] * N, steps=8)
     pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=11)
     try:
         assert pair.gpu.launch_geometry()["threads"] == 512
