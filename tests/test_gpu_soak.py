@@ -71,3 +71,48 @@ def test_random_configurations(seed):
         finally:
             tr.close()
             pair.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_looping_waves(seed):
+    """More requests than the GPU holds blocks (one resident wave of looping blocks): random row lengths (multiples of
+    four and not, so both the short loop and the general loop are taken), cache sizes, contexts on both sides of the
+    page-table staging limit, layer groups with a side-stream prefetch, policies; requests without and with misses
+    mixed at random in every launch."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rng = np.random.default_rng(seed)
+    for _ in range(5):
+        k = int(rng.choice([4, 7, 16, 33, 64, 100, 128, 256]))
+        B = int(k * rng.choice([1, 2, 3]) + rng.integers(0, 9))
+        init_len = int(rng.choice([B + 5, 3 * B, 1000, 5000, 40000]))
+        lpg = int(rng.choice([1, 1, 2]))
+        policy = int(rng.choice([hs.POLICY_LRU, hs.POLICY_LRU, hs.POLICY_FIFO, hs.POLICY_RANDOM]))
+        N = 3 * sms + int(rng.integers(1, 400))
+        w = inputs.Workload("loop", inputs.KIND_DSA_MIX, N, lpg, lpg, k, B, 16, [init_len] * N, 8)
+        pair = Pair(w, flags=hs.FLAG_DEBUG_VALIDATE, policy=policy, policy_seed=3)
+        side = torch.cuda.Stream() if lpg > 1 else None
+        try:
+            assert pair.gpu.launch_geometry()["threads"] == 512
+            for step in range(6):
+                if step % 2 == 1:
+                    pair.append()
+                rows = []
+                for r in range(N):
+                    res = pair.oracle.slot_pos(r, 0)
+                    res = res[res >= 0]
+                    if step > 0 and rng.random() < 0.6 and len(res) >= max(1, k // 2):     # nothing misses
+                        n = int(rng.integers(max(1, k // 2), min(k, len(res)) + 1))
+                        row = rng.choice(res, size=n, replace=False).astype(np.int32)
+                        if pair.oracle.newest(r) >= 0 and n < k and rng.random() < 0.5:
+                            row = np.append(row, np.int32(pair.oracle.newest(r)))
+                        row = rng.permutation(np.concatenate([row, np.full(k - len(row), -1, dtype=np.int32)]))
+                    else:
+                        row = inputs.random_rows(rng, 1, k, pair.oracle.length(r), 0.1)[0]
+                    rows.append(row)
+                rows = np.stack(rows)
+                for layer in range(lpg):
+                    pair.resolve_and_compare(layer, rows, side_stream=side)
+                    pair.compare_state(layer, requests=range(0, N, 7))
+            pair.finish()
+        finally:
+            pair.close()
