@@ -310,8 +310,20 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   if ((c->flags & HISPARSE_FLAG_NARROW_BLOCKS) && (c->flags & HISPARSE_FLAG_WIDE_BLOCKS)) return fail(HISPARSE_EINVAL);
   h->T = kThreads; h->minb = 1;
   if (want_small) {
-    for (int per_sm = 3; per_sm >= 2 && h->T == kThreads; --per_sm)   // three narrow blocks per SM if they fit, else two
-      if (try_small(per_sm)) { h->T = kThreadsSmall; h->minb = per_sm; }
+    // Three narrow blocks per SM (40 registers) only for shapes whose blocks can run the short loop (the kernel's
+    // lean_shape: one block per request, every request the same capacity, whole 16-byte rows, a page-table slice that
+    // fits the ring of a third of an SM); otherwise two (64 registers).  Measured on batches of 200 / 256 / 600
+    // C2-shaped requests, whose slices are too long to stage: with two blocks per SM a launch with misses takes
+    // 482 / 615 / 1420 us instead of 490 / 620 / 1432 and a launch without misses 12.3 / 13.3 / 23.6 us instead of
+    // 19.3 / 22.4 / 37.5; on the short loop's shapes three per SM take 61.6 us per 8192 requests instead of 65.8.
+    for (int per_sm = 3; per_sm >= 2 && h->T == kThreads; --per_sm) {
+      if (!try_small(per_sm)) continue;
+      const bool short_loop = want == 1 && d.uni_cap >= 0 && (k & 3) == 0 &&
+                              !(c->flags & (HISPARSE_FLAG_EAGER_ORDER | HISPARSE_FLAG_PHASE_TIMERS)) &&
+                              p2s_stride(d.uni_cap) * 2 + 16 <= (int64_t)d.ring_bytes;
+      if (per_sm == 3 && !short_loop) continue;
+      h->T = kThreadsSmall; h->minb = per_sm;
+    }
     if (h->T == kThreads && (c->flags & HISPARSE_FLAG_NARROW_BLOCKS)) return fail(HISPARSE_EINVAL);
   }
   if (h->T == kThreads) {
