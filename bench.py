@@ -426,8 +426,8 @@ def all_hit_points(dev, peak, sm_count):
     steady: 8192 requests, launches back to back with no flush: one launch reads and writes ~390 MB, three times L2,
             so nothing a launch touches is still cached when the next one comes to it; launch and ramp-up are
             amortised as they are in a decode loop.  This is the roofline figure.
-    flushed: 2048 requests, one launch per timing, L2 emptied (256 MiB write, then 256 MiB read) before each: the
-            survey's point; a third of its time is launch, code fetch and ramp-up of a cold kernel.
+    flushed: 2048 requests, one launch per timing, L2 emptied (256 MiB write, then 256 MiB read) before each: a
+            single cold launch; a fifth of its time is launch, code fetch and ramp-up.
     """
     import torch
     import paper_2608_07009_b200 as hs

@@ -1,7 +1,7 @@
 """The sparse-attention consumer (hisparse_sparse_attention, through the C-ABI binding) against the fp64 oracle
 (oracle/attention_oracle.py), on slot tables that the library's own resolve emitted and on hand-made ones.
 
-Tolerance (derived in the design doc): inputs are bf16 on both sides, so products are exact; the kernel accumulates in
+Tolerance: inputs are bf16 on both sides, so products are exact; the kernel accumulates in
 fp32 and rounds the softmax weights to bf16 (relative error 2^-9 each) before they multiply the values, and its
 normaliser is the sum of the unrounded weights.  out is a convex combination of the values, so
 |out - exact| <= 1e-2 * max |value| elementwise; lse is fp32 arithmetic on scores of a few units: 2e-3 absolute.
