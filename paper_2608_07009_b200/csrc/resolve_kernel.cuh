@@ -1320,6 +1320,14 @@ resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_
     __syncthreads();  // the barriers are initialised and the marks cleared before anything uses them
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (part != 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!LOOP && part == 0 && tid == 96 && r < d.N) {
+      // A request whose previous resolve on this group missed nothing will most likely miss nothing now: whatever
+      // follows in the stream may be scheduled at once, so that its launch latency and prologue run under this
+      // whole kernel instead of under its last third (a resolve that does fetch releases its dependents only once
+      // its loads are in flight: earlier costs the fetch ~2 us, which a wrong guess here pays once).  One thread of a
+      // warp that takes no part in the staging reads the flag, so nothing waits for the load.
+      if (__ldcg(d.anchor_misses + (int64_t)r * d.G + g) == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
     if (part == 0) {
       int64_t cap_r, init_len_r, p2s_off_r;
       request_geom(d, r, cap_r, init_len_r, p2s_off_r);
