@@ -1013,7 +1013,8 @@ __device__ __forceinline__ void helper_block(const DevState &d, const ReqCtx &c,
 // Same steps and same results as the general code below (lookup_phase + the short path of resolve_kernel), with
 // everything that does not depend on the request hoisted out of the loop, 32-bit lengths, and no per-request geometry
 // structs: the general code spends ~840 instructions per thread and request, which made a resolve in which nothing
-// misses issue-bound; this loop spends about a fifth of that.  A request with a miss leaves through miss_path_cold.
+// misses issue-bound; this loop spends about a fifth of that.  The first request with a miss ends the loop: the general
+// loop takes that request, and the block's later ones, from there (see lean_loop).
 __device__ __forceinline__ bool lean_shape(const DevState &d, const int32_t *sel, const int32_t *table, const int threads) {
   return !(d.flags & HISPARSE_FLAG_PHASE_TIMERS) && d.uni_cap >= 0 && d.order_t != nullptr &&
          (((uintptr_t)sel | (uintptr_t)table | (uintptr_t)d.pos2slot | (uintptr_t)d.anchor_out) & 15) == 0 &&
