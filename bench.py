@@ -637,6 +637,9 @@ def measure(args, w, dev, local, K, W, full, launched, rank):
         # ---- timed region: K graph replays, inputs resident in HBM, L2 flushed between steps ----
         step_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         launches = 0
+        in_graph = []                                                   # --phases: per-layer (start, end) of every timed step
+        if args.phases:
+            gpu.layer_times()                                           # forget the warm-up's stamps
         for s_ in range(K):
             i = 1 + W + s_
             load_step(i)
@@ -646,6 +649,8 @@ def measure(args, w, dev, local, K, W, full, launched, rank):
             step_ev[s_][1].record(main)
             save_counts(i)
             launches += launches_per_step[kv_dev[i] is not None]
+            if args.phases:
+                in_graph.append(gpu.layer_times().astype(np.int64))     # (synchronises: between steps, outside their events)
         barrier()
         clocks = sampler.stop()
 
@@ -688,6 +693,15 @@ def measure(args, w, dev, local, K, W, full, launched, rank):
                   "unit": "us, mean over requests, last anchor launch"}
         cyc = st[:, [15, 8, 9, 10, 11, 12, 13, 14]]
         phases["cycles_issue_landed_lookup_dedup_missscan_victims_ready"] = [float(x) for x in np.diff(cyc, axis=1).mean(axis=0)]
+        if in_graph:
+            # the resolve launches as they ran INSIDE the timed graph replays: the kernel's own first-request-start and
+            # last-request-end stamps per layer, and the gaps between consecutive launches
+            ig = np.stack(in_graph)[:, [l for l in range(L) if l % lpg == 0], :]
+            dur = (ig[:, :, 1] - ig[:, :, 0]) / 1e3
+            gap = (ig[:, 1:, 0] - ig[:, :-1, 1]) / 1e3 if ig.shape[1] > 1 else np.zeros((1, 1))
+            phases["in_graph_launch_us"] = {"median": float(np.median(dur)), "p99": float(np.percentile(dur, 99)),
+                                            "mean": float(dur.mean()), "launches": int(dur.size)}
+            phases["in_graph_gap_us"] = {"median": float(np.median(gap)), "p99": float(np.percentile(gap, 99))}
         out["phases"] = phases
 
     if full:

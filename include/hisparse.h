@@ -263,6 +263,12 @@ int hisparse_device_bytes(const hisparse_config_t *cfg, size_t *kv_bytes, size_t
  * classified, [11] / [12] counted, before / after the barrier, [13] scanned, [14] plan ready.  Synchronises. */
 int hisparse_phase_times(hisparse_t *h, uint64_t *out);
 
+/* With PHASE_TIMERS: for every layer, when its last resolve kernel started its first request and finished its last
+ * one (%globaltimer nanoseconds; host uint64 [2][L]: the L starts, then the L ends; a layer that was not resolved
+ * since the last call reads start = UINT64_MAX, end = 0).  Inside a CUDA-graph replay of a whole step this gives the
+ * duration of each launch and the gaps between launches without a profiler.  Synchronises, then clears the stamps. */
+int hisparse_layer_times(hisparse_t *h, uint64_t *out);
+
 /* Failure-detection self-test.  Every device-side wait of the library (on the mbarriers of its bulk copies) is
  * bounded: after 2 s it gives up, sets STATUS_TIMEOUT and the kernel returns, so a lost completion can never hang
  * the GPU.  This call runs that very wait on a barrier that nothing completes, with a limit of limit_ns

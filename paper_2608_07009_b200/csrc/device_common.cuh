@@ -66,6 +66,7 @@ struct DevState {
   int policy;                      // HISPARSE_POLICY_*
   unsigned long long policy_seed;  // RANDOM policy
   unsigned long long *phase_ns;    // [N][16]: 8 globaltimer stamps, then 8 SM cycle-counter stamps (PHASE_TIMERS)
+  unsigned long long *layer_ns;    // [2][L]: earliest request start / latest request end of each layer's last resolve (PHASE_TIMERS)
 };
 
 // ------------------------------------------------------------------------------------------ device helpers

@@ -392,6 +392,7 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRY(dev_alloc(h, &h->hint_hits, (size_t)N));
   HS_TRY(dev_alloc(h, &h->hint_misses, (size_t)N));
   HS_TRY(dev_alloc(h, &d.phase_ns, (size_t)N * 16));
+  HS_TRY(dev_alloc(h, &d.layer_ns, (size_t)L * 2));
 #undef HS_TRY
   d.cap = h->d_cap; d.init_len = h->d_init_len; d.p2s_off = h->d_p2s_off; d.host = h->d_host;
 
@@ -414,6 +415,8 @@ int hisparse_create(const hisparse_config_t *c, hisparse_t **out) {
   HS_TRYC(cudaMemset(d.ticket, 0, 4));
   HS_TRYC(cudaMemset(d.status, 0, 4));
   HS_TRYC(cudaMemset(d.phase_ns, 0, (size_t)N * 16 * 8));
+  HS_TRYC(cudaMemset(d.layer_ns, 0xff, (size_t)L * 8));
+  HS_TRYC(cudaMemset(d.layer_ns + L, 0, (size_t)L * 8));
   init_order_kernel<<<296, 256>>>(d.order, (int64_t)NG * B, B);
   HS_TRYC(cudaGetLastError());
 
@@ -786,6 +789,17 @@ int hisparse_phase_times(hisparse_t *h, uint64_t *out) {
   HS_CUDA(cudaSetDevice(h->device));
   HS_CUDA(cudaDeviceSynchronize());
   HS_CUDA(cudaMemcpy(out, h->d.phase_ns, (size_t)h->d.N * 16 * 8, cudaMemcpyDeviceToHost));
+  return HISPARSE_OK;
+}
+
+int hisparse_layer_times(hisparse_t *h, uint64_t *out) {
+  if (!h || !out) return HISPARSE_EINVAL;
+  const size_t L = (size_t)h->d.L;
+  HS_CUDA(cudaSetDevice(h->device));
+  HS_CUDA(cudaDeviceSynchronize());
+  HS_CUDA(cudaMemcpy(out, h->d.layer_ns, L * 2 * 8, cudaMemcpyDeviceToHost));
+  HS_CUDA(cudaMemset(h->d.layer_ns, 0xff, L * 8));   // start = "none yet"
+  HS_CUDA(cudaMemset(h->d.layer_ns + L, 0, L * 8));
   return HISPARSE_OK;
 }
 

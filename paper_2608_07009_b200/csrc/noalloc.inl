@@ -89,6 +89,7 @@ int hisparse_resolve_noalloc(const hisparse_external_state_t *st, const int32_t 
   d.status = status_dev ? status_dev : reinterpret_cast<uint32_t *>(scratch + 2 * kNoAllocPlanBytes + 3 * kNoAllocCounterBytes);
   d.ticket = nullptr;
   d.phase_ns = nullptr;      // only touched with PHASE_TIMERS, which is off here
+  d.layer_ns = nullptr;
   layout_smem(d, kThreads, true, false);   // a request's two blocks may share the page-table lookups
   if (!layout_ring(d, kThreads, (int64_t)optin - 1024 - d.meta_smem - d.bar_bytes)) return HISPARSE_EINVAL;
   const size_t smem = kernel_smem_bytes(d);

@@ -952,6 +952,7 @@ __device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, co
       const unsigned long long now = global_ns();
       stamps[5] = now;
       atomicMax(&stamps[6], now);
+      atomicMax(d.layer_ns + d.L + c.layer, now);
     }
   }
 }
@@ -1004,7 +1005,11 @@ __device__ __forceinline__ void helper_block(const DevState &d, const ReqCtx &c,
   fetch_parity = fetch.parity;
   if (d.flags & HISPARSE_FLAG_PHASE_TIMERS) {
     __syncthreads();
-    if (tid == 0) atomicMax(&d.phase_ns[(int64_t)c.r * 16 + 6], global_ns());
+    if (tid == 0) {
+      const unsigned long long now = global_ns();
+      atomicMax(&d.phase_ns[(int64_t)c.r * 16 + 6], now);
+      atomicMax(d.layer_ns + d.L + c.layer, now);
+    }
   }
 }
 
@@ -1363,7 +1368,10 @@ resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_
     const SmemView v = smem_view(d, smem_raw, it);
     const SliceGeom q = slice_geom(d, g, c.cap_r, c.p2s_off_r);
     unsigned long long *stamps = d.phase_ns + (int64_t)r * 16;
-    if (timers && tid == 0) { stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64(); }
+    if (timers && tid == 0) {
+      stamps[0] = global_ns(); stamps[6] = 0ull; stamps[15] = clock64();
+      atomicMin(d.layer_ns + layer, stamps[0]);
+    }
     c.tag = it % 255 + 1;
     if (LOOP && it > 0 && c.tag == 1) {
       // the tags start over: forget the old marks (every thread is done with the previous request's)
@@ -1456,7 +1464,7 @@ resolve_kernel(const __grid_constant__ DevState d, const int layer, const int32_
       d.plan_n[c.rg] = 0;
       d.t[c.rg] = t;
       if (d.policy == HISPARSE_POLICY_FIFO) d.order_t[c.rg] = t;
-      if (timers) stamps[4] = global_ns();
+      if (timers) { stamps[4] = global_ns(); atomicMax(d.layer_ns + d.L + layer, stamps[4]); }
     }
     if (my_status) atomicOr(d.status, my_status);
     if (S > 1) {  // the other blocks of the cluster find an empty plan

@@ -26,7 +26,7 @@ EXPORTS = [
     "hisparse_create", "hisparse_destroy", "hisparse_append", "hisparse_resolve", "hisparse_prefetch", "hisparse_prefetch_hint",
     "hisparse_join", "hisparse_layer_pool", "hisparse_gather", "hisparse_gather_check", "hisparse_status",
     "hisparse_clear_status", "hisparse_dump_state", "hisparse_order_lag", "hisparse_load_state", "hisparse_load_appends", "hisparse_dump_plan", "hisparse_device_bytes",
-    "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_selftest_wait_timeout", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
+    "hisparse_launch_geometry", "hisparse_phase_times", "hisparse_layer_times", "hisparse_selftest_wait_timeout", "hisparse_host_alloc", "hisparse_host_free", "hisparse_host_link_probe",
     "hisparse_scatter_read_probe", "hisparse_resolve_noalloc", "hisparse_strerror", "hisparse_last_cuda_error",
     "hisparse_attention_workspace_bytes", "hisparse_sparse_attention",
 ]
@@ -97,6 +97,7 @@ def lib() -> ctypes.CDLL:
             "hisparse_device_bytes": ([P(Config), P(sz), P(sz)], i32),
             "hisparse_launch_geometry": ([vp, P(ctypes.c_int32), P(ctypes.c_int32), P(ctypes.c_int32)], i32),
             "hisparse_phase_times": ([vp, vp], i32),
+            "hisparse_layer_times": ([vp, vp], i32),
             "hisparse_selftest_wait_timeout": ([vp, ctypes.c_uint64, P(ctypes.c_uint64)], i32),
             "hisparse_host_alloc": ([sz, P(vp)], i32),
             "hisparse_host_free": ([vp], i32),
@@ -367,6 +368,13 @@ class HiSparse:
         out = np.zeros((self.N, 16), dtype=np.uint64)
         _check(lib().hisparse_phase_times(self._h, out.ctypes.data), "hisparse_phase_times")
         return out
+
+    def layer_times(self) -> np.ndarray:
+        """uint64 [L][2]: start and end (ns) of each layer's last resolve kernel since the previous call (needs
+        FLAG_PHASE_TIMERS); a layer without one reads (2**64 - 1, 0).  Synchronises and clears the stamps."""
+        out = np.zeros((2, self.L), dtype=np.uint64)
+        _check(lib().hisparse_layer_times(self._h, out.ctypes.data), "hisparse_layer_times")
+        return np.ascontiguousarray(out.T)
 
     def selftest_wait_timeout(self, limit_ns: int) -> int:
         """Runs the library's bounded wait on a barrier that never completes; returns the nanoseconds waited."""

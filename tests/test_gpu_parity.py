@@ -648,6 +648,30 @@ def test_bounded_wait_expires_and_the_handle_stays_usable():
 
 # ------------------------------------------------------------------ boundary errors
 
+def test_layer_times_bracket_every_resolve():
+    """With PHASE_TIMERS every anchor resolve leaves its start and end stamps per layer; layers resolved one after the
+    other on a stream are ordered in time; reading clears the stamps."""
+    w = inputs.c2_dsa_decode(num_requests=3, num_layers=4, steps=3, context=3000)
+    pair = Pair(w, flags=hs.FLAG_PHASE_TIMERS)
+    tr = inputs.Trace(w)
+    try:
+        sel, appended, _ = tr.step()
+        if appended:
+            pair.append()
+        for layer in range(4):
+            pair.resolve_and_compare(layer, sel[layer])
+        lt = pair.gpu.layer_times().astype(np.int64)
+        assert lt.shape == (4, 2)
+        assert np.all(lt[:, 1] > lt[:, 0]) and np.all(lt[:, 1] - lt[:, 0] < 10_000_000)
+        assert np.all(lt[1:, 0] >= lt[:-1, 1])
+        cleared = pair.gpu.layer_times()
+        assert np.all(cleared[:, 0] == np.uint64(2**64 - 1)) and np.all(cleared[:, 1] == 0)
+        pair.finish()
+    finally:
+        tr.close()
+        pair.close()
+
+
 def test_create_rejects_bad_arguments():
     hist = HostHistory(1, 64, 32)
     try:
