@@ -54,7 +54,12 @@ typedef struct hisparse hisparse_t; /* opaque, library-owned */
 #define HISPARSE_FLAG_PHASE_TIMERS 8u      /* the resolve kernel records %globaltimer at its phase boundaries
                                              (hisparse_phase_times); for the phase breakdown of Fig. 7        */
 
-#define HISPARSE_FLAG_NO_PDL 16u           /* launch Resolve without programmatic dependent launch             */
+#define HISPARSE_FLAG_NO_PDL 16u           /* launch Resolve without programmatic dependent launch.  By default the
+                                             kernel waits for its predecessor in the stream with
+                                             griddepcontrol.wait and lets its own successor be scheduled early; a
+                                             successor that the caller launches with programmatic stream
+                                             serialization must itself wait for the grid dependency before it reads
+                                             what Resolve wrote (kernels launched the ordinary way are unaffected)  */
 
 #define HISPARSE_FLAG_EAGER_ORDER 32u      /* bring the recency list up to date in every Resolve.  By default a
                                              Resolve in which nothing missed only stamps its hits (the stamps of
