@@ -821,7 +821,7 @@ def measure(args, w, dev, local, K, W, full, launched, rank):
         hb = min(hist[0].nbytes, 1 << 32)
         sm_count = torch.cuda.get_device_properties(local).multi_processor_count
         out["sm_read"] = {"%dMB" % mb: hs.scatter_read_probe(hist[0].ptr, hb, E, max(1, (mb << 20) // E), sm_count, 5, local)
-                          for mb in (4, 32)}
+                          for mb in (2, 4, 32)}
     del graphs
     gpu.close()
     for h in hist:
