@@ -793,14 +793,6 @@ __device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, co
   unsigned long long *stamps = d.phase_ns + (int64_t)r * 16;
   int *s_misc = v.misc;
   int m = 0, n_nonhit = 0;
-  for (int i = tid; i < W; i += T) v.vicbits[i] = 0u;  // ordered before their first use by list_misses' barriers
-  // the hit marks as a bitset, which the victim choice and the list rewrite work on (every mark was written before
-  // the vote; the loop bound is uniform, so every lane takes part in the ballot)
-  for (int sb = 0; sb < B; sb += T) {
-    const int s = sb + tid;
-    const uint32_t word = __ballot_sync(0xffffffffu, s < B && v.marks[s] == (uint8_t)c.tag);
-    if (lane == 0 && (s >> 5) < W) v.hitbits[s >> 5] = word;
-  }
   // The recency list starts its way into the memory the row occupied (every thread consumed its row entries before
   // the vote); it is needed only once the first loads are in flight.
   const uint16_t *order_g = d.order + rg * B;
@@ -823,6 +815,16 @@ __device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, co
   TmaFetch fetch;
   fetch.init(d, r, c.layer, m, v.plan_pos, v.plan_slot, v.ring, v.bars, 0, S, fetch_parity);
   fetch.issue(d);
+  // With the loads on their way: the victim marks cleared and the hit marks turned into a bitset, which the victim
+  // choice and the list rewrite work on (every mark was written before the vote; the loop bound is uniform, so
+  // every lane takes part in the ballot).  Both are ordered before their first use by choose_victims' barrier.
+  // (Before the loads, this cost the fetch 1100 cycles of waiting.)
+  for (int i = tid; i < W; i += T) v.vicbits[i] = 0u;
+  for (int sb = 0; sb < B; sb += T) {
+    const int s = sb + tid;
+    const uint32_t word = __ballot_sync(0xffffffffu, s < B && v.marks[s] == (uint8_t)c.tag);
+    if (lane == 0 && (s >> 5) < W) v.hitbits[s >> 5] = word;
+  }
 #define HS_VICT(IPT) choose_victims<T, IPT>(d, v, r, rg, m, stamps, t, order_t, order_bulk, order_parity, my_status, n_nonhit)
   if constexpr (T == kThreads) {
     if (B <= 4 * T) HS_VICT(4);
