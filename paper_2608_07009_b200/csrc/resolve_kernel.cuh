@@ -793,6 +793,14 @@ __device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, co
   unsigned long long *stamps = d.phase_ns + (int64_t)r * 16;
   int *s_misc = v.misc;
   int m = 0, n_nonhit = 0;
+  int16_t *s_p2s = reinterpret_cast<int16_t *>(v.ring) + slice_geom(d, c.g, c.cap_r, c.p2s_off_r).lead;
+  list_misses<T, KPT>(d, v, c.trow, c.arow, stamps, s_misc, s_p2s, claims, pos, cls, my_status, m);
+  if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
+  // Phase 4 starts here, with the positions of the misses: the first batch of host loads is in flight while the
+  // victims are chosen (a record's slot is only needed when it is stored) and the metadata is written back
+  TmaFetch fetch;
+  fetch.init(d, r, c.layer, m, v.plan_pos, v.plan_slot, v.ring, v.bars, 0, S, fetch_parity);
+  fetch.issue(d);
   // The recency list starts its way into the memory the row occupied (every thread consumed its row entries before
   // the vote); it is needed only once the first loads are in flight.
   const uint16_t *order_g = d.order + rg * B;
@@ -807,14 +815,6 @@ __device__ __forceinline__ void miss_path(const DevState &d, const ReqCtx &c, co
   } else {
     stage_async(v.order, order_g, B * 2);
   }
-  int16_t *s_p2s = reinterpret_cast<int16_t *>(v.ring) + slice_geom(d, c.g, c.cap_r, c.p2s_off_r).lead;
-  list_misses<T, KPT>(d, v, c.trow, c.arow, stamps, s_misc, s_p2s, claims, pos, cls, my_status, m);
-  if (timers && tid == 0) { stamps[3] = global_ns(); stamps[7] = stamps[3]; }
-  // Phase 4 starts here, with the positions of the misses: the first batch of host loads is in flight while the
-  // victims are chosen (a record's slot is only needed when it is stored) and the metadata is written back
-  TmaFetch fetch;
-  fetch.init(d, r, c.layer, m, v.plan_pos, v.plan_slot, v.ring, v.bars, 0, S, fetch_parity);
-  fetch.issue(d);
   // With the loads on their way: the victim marks cleared and the hit marks turned into a bitset, which the victim
   // choice and the list rewrite work on (every mark was written before the vote; the loop bound is uniform, so
   // every lane takes part in the ballot).  Both are ordered before their first use by choose_victims' barrier.
